@@ -1,0 +1,277 @@
+"""CPU checker for the verification step of judge decoding (arXiv 2501.19309).
+
+TEST INFRASTRUCTURE ONLY.  This is a plain, slow, float64 restatement of what
+one verification call computes, written from the paper so that a reader can
+check it by eye.  Nothing in the product may import it: only the tests, the
+smoke check and the CPU-baseline leg of the benchmark do.  It shares no code
+with the CUDA library and never sees a value the CUDA library produced.
+
+What one call computes (paper Sec. 3.1 "Speculative decoding", Eq. 2-4, and
+Sec. 4.1 "Inference"; 0-indexed here, the paper is 1-indexed):
+
+  for every sequence b and every row j = 0..M of its embeddings H[b]:
+      L[j, :] = W @ H[b, j]                      LM head (Eq. 2)
+      p_j     = softmax(L[j, :])                 target distribution of slot j
+  for every draft slot j = 0..M-1 with drafted token x_j:
+      q_j     = softmax(draft_logits[b, j, :])   draft distribution (Eq. 3)
+      z_std[j]   = u_j * q_j[x_j] < p_j[x_j]     standard test (Eq. 4)
+      s[j]       = sigmoid(w . H[b, j+1] + b0)   judge score of x_j's own embedding
+      z_judge[j] = s[j] > tau                    (Sec. 4.1 "Inference")
+      z[j]       = z_std[j] or z_judge[j]        (or one of them, by mode)
+  a = index of the first j with z[j] == 0, else M   ("if all previous tokens are accepted")
+  next token: from the residual max(0, p_a - q_a), normalised, when a < M;
+              from p_M after a fully accepted block; inverse CDF in ascending
+              token id with one uniform.
+
+Readings taken where the paper is silent (all restated in the design notes):
+  * the judge for draft token j reads row j+1 of H, the embedding produced by
+    feeding that token (Sec. 4.1 speaks of the embedding of the current token);
+  * the token at the first rejection comes from the residual distribution, the
+    form that keeps standard speculative sampling lossless; the paper's literal
+    "sample from p_i" is available as resample="target_p";
+  * Eq. 4 is evaluated division-free, u*q < p, which equals u < min(1, p/q)
+    for u in [0, 1); q(x) = 0 accepts iff p(x) > 0;
+  * the judge comparison is strict; tau = 1 never accepts, so the OR mode
+    reduces to the standard test (Sec. 4.1, last sentence);
+  * uniforms: Philox4x32-10 (Salmon et al., SC'11), key = the 64-bit seed split
+    in two words, counter = (b, slot, stream, 0), first output word, top 24
+    bits: u = (word >> 8) * 2**-24.  stream 0 feeds the acceptance test of slot
+    j, stream 1 the token draw at slot a;
+  * an all-zero residual (p_a == q_a) falls back to sampling from p_a;
+  * inverse CDF: T = u' * sum(r); token = min{t : r[0] + .. + r[t] > T}; if
+    rounding leaves no such t, the last token with r > 0.
+
+Pins (tests/test_oracle_*.py): Philox known-answer vectors printed with the
+generator's publication; closed forms of the acceptance law and of the emitted
+token law by exhaustive enumeration on tiny vocabularies; q = p accepts all;
+tau = 1 and mode "standard" equal a separate textbook routine; chi-square of the
+emitted token against p; judge special cases (w = 0, w = unit vector); the
+prefix rule over all 2^M masks; OR monotonicity; one-hot residuals.
+Parity unpinned: nothing about real-model behaviour (acceptance lengths or
+accuracy with trained weights) is checked anywhere.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Optional, Sequence
+
+import numpy as np
+
+MODE_STANDARD, MODE_JUDGE, MODE_JUDGE_OR_STANDARD = 0, 1, 2
+RESAMPLE_RESIDUAL, RESAMPLE_TARGET_P = 0, 1
+STREAM_ACCEPT, STREAM_SAMPLE = 0, 1
+
+_MODES = {"standard": MODE_STANDARD, "judge": MODE_JUDGE, "judge_or_standard": MODE_JUDGE_OR_STANDARD}
+_RESAMPLE = {"residual": RESAMPLE_RESIDUAL, "target_p": RESAMPLE_TARGET_P}
+
+
+# --------------------------------------------------------------------------
+# Philox4x32-10, from its published definition (Salmon, Moraes, Dror, Shaw:
+# "Parallel random numbers: as easy as 1, 2, 3", SC'11, Sec. 3.3 / Table 2).
+# --------------------------------------------------------------------------
+_PHILOX_M0 = 0xD2511F53
+_PHILOX_M1 = 0xCD9E8D57
+_PHILOX_W0 = 0x9E3779B9   # golden ratio
+_PHILOX_W1 = 0xBB67AE85   # sqrt(3) - 1
+_MASK32 = 0xFFFFFFFF
+
+
+def philox4x32_10(counter: Sequence[int], key: Sequence[int]) -> tuple:
+    """One Philox4x32-10 block: 4 counter words, 2 key words -> 4 output words."""
+    c0, c1, c2, c3 = (int(c) & _MASK32 for c in counter)
+    k0, k1 = (int(k) & _MASK32 for k in key)
+    for rnd in range(10):
+        if rnd > 0:                      # the key is bumped between rounds (9 bumps)
+            k0 = (k0 + _PHILOX_W0) & _MASK32
+            k1 = (k1 + _PHILOX_W1) & _MASK32
+        prod0 = _PHILOX_M0 * c0          # 64-bit products
+        prod1 = _PHILOX_M1 * c2
+        hi0, lo0 = prod0 >> 32, prod0 & _MASK32
+        hi1, lo1 = prod1 >> 32, prod1 & _MASK32
+        c0, c1, c2, c3 = hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0
+    return c0, c1, c2, c3
+
+
+def uniform24(seed: int, b: int, slot: int, stream: int) -> float:
+    """u in [0, 1) on the 2**-24 grid, keyed by (seed; b, slot, stream)."""
+    key = (seed & _MASK32, (seed >> 32) & _MASK32)
+    word0 = philox4x32_10((b, slot, stream, 0), key)[0]
+    return (word0 >> 8) * 2.0 ** -24
+
+
+# --------------------------------------------------------------------------
+# storage widening (own copy: the checker shares no helper with anything else)
+# --------------------------------------------------------------------------
+def _to_f64(a: np.ndarray) -> np.ndarray:
+    """float64 values of a stored array: uint16 = bfloat16 bit patterns, else floats."""
+    a = np.asarray(a)
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    return a.astype(np.float64)
+
+
+# --------------------------------------------------------------------------
+# the steps
+# --------------------------------------------------------------------------
+def project_logits(W: np.ndarray, Hb: np.ndarray, vocab_chunk: int = 8192) -> np.ndarray:
+    """L[j, v] = sum_k H[j, k] * W[v, k] in float64 (Eq. 2, LM head).
+
+    W is widened to float64 a slab of vocabulary rows at a time only to bound
+    memory; every L[j, v] is still one full-length dot product."""
+    Hd = _to_f64(Hb)                                    # [rows, d]
+    V = W.shape[0]
+    L = np.empty((Hd.shape[0], V), dtype=np.float64)
+    for v0 in range(0, V, vocab_chunk):
+        v1 = min(V, v0 + vocab_chunk)
+        L[:, v0:v1] = Hd @ _to_f64(W[v0:v1]).T
+    return L
+
+
+def logsumexp(row: np.ndarray) -> tuple:
+    """(max, log sum exp) of one row, float64."""
+    m = float(np.max(row))
+    return m, m + float(np.log(np.sum(np.exp(row - m))))
+
+
+def sigmoid(t: float) -> float:
+    return 1.0 / (1.0 + float(np.exp(-t)))
+
+
+def accepted_prefix_length(z: Sequence[int]) -> int:
+    """Index of the first rejected slot, or len(z) when every slot is accepted."""
+    for j, zj in enumerate(z):
+        if not zj:
+            return j
+    return len(z)
+
+
+def combine_masks(z_std: int, z_judge: int, mode: int) -> int:
+    if mode == MODE_STANDARD:
+        return int(z_std)
+    if mode == MODE_JUDGE:
+        return int(z_judge)
+    return int(z_std or z_judge)
+
+
+def inverse_cdf(r: np.ndarray, u: float) -> tuple:
+    """token = min{t : r[0]+..+r[t] > u * sum(r)}; returns (token, T, cdf)."""
+    cdf = np.cumsum(r, dtype=np.float64)                # sequential float64 prefix sums
+    total = float(cdf[-1])
+    T = u * total
+    t = int(np.searchsorted(cdf, T, side="right"))      # first index with cdf > T
+    if t >= len(r):                                      # rounding: take the last token with mass
+        t = int(np.max(np.nonzero(r > 0)[0]))
+    return t, T, cdf
+
+
+@dataclasses.dataclass
+class OracleResult:
+    sequences: list                 # which b were computed (all by default)
+    accept_len: np.ndarray          # [B] int32 (-1 where not computed)
+    next_token: np.ndarray          # [B] int32 (-1 where not computed)
+    judge_scores: np.ndarray        # [B, M] float64
+    p_draft: np.ndarray             # [B, M] float64  p_j[x_j]
+    q_draft: np.ndarray             # [B, M] float64  q_j[x_j]
+    masks: np.ndarray               # [B, M] uint8: bit0 standard test, bit1 judge test
+    row_max: np.ndarray             # [B, M+1] float64  max_v L
+    row_lse: np.ndarray             # [B, M+1] float64  logsumexp_v L
+    u_accept: np.ndarray            # [B, M] float64 uniforms of the acceptance test
+    u_sample: np.ndarray            # [B] float64 uniform of the token draw
+    margin_accept: np.ndarray       # [B, M] |u - min(1, p/q)|
+    margin_judge: np.ndarray        # [B, M] |s - tau|
+    margin_cdf: np.ndarray          # [B] distance of T to the nearest CDF edge of the token, / sum(r)
+    sample_T: np.ndarray            # [B] T = u' * sum(r)
+    sample_mass: np.ndarray         # [B] sum(r)
+    sample_weights: dict            # b -> r[V] float64 (un-normalised sampling weights)
+    logits: dict                    # b -> L[M+1, V] float64 (kept only when keep_logits)
+
+    def token_interval(self, b: int, token: int) -> tuple:
+        """CDF interval [lo, hi) of ``token`` in sequence b's sampling weights."""
+        r = self.sample_weights[b]
+        cdf = np.cumsum(r, dtype=np.float64)
+        lo = float(cdf[token - 1]) if token > 0 else 0.0
+        return lo, float(cdf[token])
+
+
+def jd_oracle_verify(W, w_judge, b_judge: float, H, draft_tokens, draft_logits, tau: float,
+                     seed: int, mode="judge_or_standard", resample="residual",
+                     sequences: Optional[Sequence[int]] = None, keep_logits: bool = False,
+                     u_accept: Optional[np.ndarray] = None,
+                     u_sample: Optional[np.ndarray] = None) -> OracleResult:
+    """One verification call, step by step, in float64.
+
+    ``u_accept`` [B, M] / ``u_sample`` [B], when given, replace the Philox
+    uniforms (used by the enumeration tests, which sweep u over a dyadic grid).
+    ``sequences`` restricts the work to some b (sampled checks at full size)."""
+    mode = _MODES[mode] if isinstance(mode, str) else int(mode)
+    resample = _RESAMPLE[resample] if isinstance(resample, str) else int(resample)
+    H = np.asarray(H)
+    B, Mp1, d = H.shape
+    M = Mp1 - 1
+    x = np.asarray(draft_tokens).reshape(B, M)
+    dl = np.asarray(draft_logits).reshape(B, M, -1)
+    V = W.shape[0]
+    wj = _to_f64(w_judge)
+    seqs = list(range(B)) if sequences is None else list(sequences)
+
+    res = OracleResult(
+        sequences=seqs,
+        accept_len=np.full(B, -1, np.int32), next_token=np.full(B, -1, np.int32),
+        judge_scores=np.full((B, M), np.nan), p_draft=np.full((B, M), np.nan),
+        q_draft=np.full((B, M), np.nan), masks=np.zeros((B, M), np.uint8),
+        row_max=np.full((B, M + 1), np.nan), row_lse=np.full((B, M + 1), np.nan),
+        u_accept=np.full((B, M), np.nan), u_sample=np.full(B, np.nan),
+        margin_accept=np.full((B, M), np.nan), margin_judge=np.full((B, M), np.nan),
+        margin_cdf=np.full(B, np.nan), sample_T=np.full(B, np.nan), sample_mass=np.full(B, np.nan),
+        sample_weights={}, logits={})
+
+    for b in seqs:
+        Hb = _to_f64(H[b])                               # [M+1, d]
+        L = project_logits(W, H[b])                      # [M+1, V]          (Eq. 2)
+        lse_p = np.empty(M + 1)
+        for j in range(M + 1):
+            res.row_max[b, j], lse_p[j] = logsumexp(L[j])
+        res.row_lse[b] = lse_p
+
+        lse_q = np.empty(M)
+        z = []
+        for j in range(M):
+            dlj = dl[b, j].astype(np.float64)
+            _, lse_q[j] = logsumexp(dlj)                                    # (Eq. 3: q_j)
+            xj = int(x[b, j])
+            P = float(np.exp(L[j, xj] - lse_p[j]))                          # p_j[x_j]
+            Q = float(np.exp(dlj[xj] - lse_q[j]))                           # q_j[x_j]
+            u = float(u_accept[b, j]) if u_accept is not None else uniform24(seed, b, j, STREAM_ACCEPT)
+            z_std = int(u * Q < P)                                          # (Eq. 4)
+            s = sigmoid(float(wj @ Hb[j + 1]) + b_judge)                    # judge on x_j's embedding
+            z_judge = int(s > tau)                                          # (Sec. 4.1)
+            z.append(combine_masks(z_std, z_judge, mode))
+            res.p_draft[b, j], res.q_draft[b, j], res.judge_scores[b, j] = P, Q, s
+            res.masks[b, j] = z_std | (z_judge << 1)
+            res.u_accept[b, j] = u
+            ratio = 1.0 if Q == 0.0 else min(1.0, P / Q)
+            res.margin_accept[b, j] = abs(u - ratio)
+            res.margin_judge[b, j] = abs(s - tau)
+
+        a = accepted_prefix_length(z)                                       # prefix rule
+        res.accept_len[b] = a
+
+        p_a = np.exp(L[a] - lse_p[a])
+        if a < M and resample == RESAMPLE_RESIDUAL:
+            q_a = np.exp(dl[b, a].astype(np.float64) - lse_q[a])
+            r = np.maximum(0.0, p_a - q_a)
+            if not np.any(r > 0):                                           # p_a == q_a
+                r = p_a
+        else:
+            r = p_a                                                         # bonus token, or literal reading
+        u2 = float(u_sample[b]) if u_sample is not None else uniform24(seed, b, a, STREAM_SAMPLE)
+        t, T, cdf = inverse_cdf(r, u2)
+        res.next_token[b] = t
+        res.u_sample[b] = u2
+        res.sample_T[b], res.sample_mass[b] = T, float(cdf[-1])
+        lo = float(cdf[t - 1]) if t > 0 else 0.0
+        res.margin_cdf[b] = min(abs(T - lo), abs(float(cdf[t]) - T)) / float(cdf[-1])
+        res.sample_weights[b] = r
+        if keep_logits:
+            res.logits[b] = L
+    return res

@@ -1,0 +1,165 @@
+/*
+ * jd.h - C ABI of the judge-decoding verification step for NVIDIA B200 (sm_100a).
+ *
+ * One call, jd_verify, performs what follows every target-model forward over a block of M
+ * draft tokens in judge decoding (arXiv 2501.19309):
+ *   1. LM-head projection of the target's last-layer embeddings, L = H W^T      (Sec. 3.1, Eq. 2)
+ *   2. softmax over the vocabulary, p_j = softmax(L[j,:]), and q_j = softmax(draft logits)
+ *   3. the standard speculative-sampling test u_j q_j[x_j] < p_j[x_j]            (Sec. 3.1, Eq. 4)
+ *      and the judge test sigmoid(w . H[b,j+1] + b0) > tau                      (Sec. 4.1 "Inference")
+ *   4. mask = standard OR judge (or one of them), accepted prefix length        (Sec. 4.1; App. B.2)
+ *   5. the next token: from normalised max(0, p - q) at the first rejection, from the extra
+ *      row p_M after a fully accepted block                                     (Sec. 3.1, after Eq. 4)
+ * The logits exist only on chip; they are never written to device memory unless the
+ * test-only logits_debug pointer is set.
+ *
+ * Conventions
+ *   - Indices are 0-based. Row j of H[b] (j = 0..M) yields p_j, the target distribution of draft
+ *     slot j; row 0 belongs to the last context token, row j >= 1 to draft token j-1. The judge
+ *     score of draft token j is read from row j+1. Row M also yields the bonus distribution.
+ *   - All tensors are dense, row-major (last index fastest).
+ *   - Unless a function says "host", every data pointer is a DEVICE pointer owned by the caller.
+ *     The library never frees or keeps caller memory, except that W and w_judge given to
+ *     jd_set_head are borrowed until the next jd_set_head or jd_destroy.
+ *   - jd_verify is asynchronous on the given CUDA stream and never synchronises it.
+ *   - No function throws, prints or exits; every failure is a jd_status_t.
+ *   - Uniforms: Philox4x32-10, key = (seed low word, seed high word), counter =
+ *     (b, slot, stream, 0), first output word, u = (word >> 8) * 2^-24. stream 0 is the
+ *     acceptance draw of slot j, stream 1 the token draw at slot accept_len[b].
+ */
+#ifndef JD_H_
+#define JD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  JD_OK = 0,
+  JD_ERR_INVALID_ARG = 1, /* null pointer, size out of range, bad enum, misaligned pointer */
+  JD_ERR_UNSUPPORTED = 2, /* shape or dtype that no kernel variant covers */
+  JD_ERR_ARCH = 3,        /* the current device is not compute capability 10.x */
+  JD_ERR_ALLOC = 4,       /* device or host allocation failed */
+  JD_ERR_CUDA = 5,        /* a CUDA runtime or driver call failed */
+  JD_ERR_TIMEOUT = 6,     /* device status: a bounded wait inside a kernel ran out */
+  JD_ERR_BAD_TOKEN = 7    /* device status: a draft token was outside [0, V) and was clamped */
+} jd_status_t;
+
+typedef enum { JD_DTYPE_F32 = 0, JD_DTYPE_BF16 = 1 } jd_dtype_t;
+
+/* Which tests form the accept mask (Sec. 4.1 "Inference"): the standard test alone (Eq. 4),
+ * the judge alone, or their logical OR (the paper's judge decoding). */
+typedef enum { JD_MODE_STANDARD = 0, JD_MODE_JUDGE = 1, JD_MODE_JUDGE_OR_STANDARD = 2 } jd_mode_t;
+
+/* Distribution of the token drawn at the first rejected slot a < M.
+ * RESIDUAL: normalised max(0, p_a - q_a), the form under which the standard test is lossless;
+ *           an identically zero residual falls back to p_a.
+ * TARGET_P: p_a itself, the literal wording of Sec. 3.1 ("sample a correct token from p_i").
+ * After a fully accepted block the token always comes from p_M. */
+typedef enum { JD_RESAMPLE_RESIDUAL = 0, JD_RESAMPLE_TARGET_P = 1 } jd_resample_t;
+
+/* Kernel family used by jd_verify. AUTO picks the fastest one that supports the shape. */
+typedef enum {
+  JD_VARIANT_AUTO = 0,
+  JD_VARIANT_SIMT = 1,   /* CUDA-core reference pipeline: any shape, f32 or bf16 */
+  JD_VARIANT_FUSED = 2,  /* one persistent tcgen05/TMA kernel, logits parked in tensor memory;
+                            bf16, d % 64 == 0, B*(M+1) <= 80, V <= 7*128*(number of SMs) */
+  JD_VARIANT_BATCHED = 3 /* tcgen05 GEMM with fused statistics + second pass over the selected
+                            rows; bf16, d % 64 == 0, any number of rows */
+} jd_variant_t;
+
+typedef struct {
+  int32_t max_B;    /* largest number of sequences per call, >= 1 */
+  int32_t max_M;    /* largest number of draft tokens per sequence, >= 1 */
+  int32_t d;        /* embedding width */
+  int32_t V;        /* vocabulary size */
+  int32_t dtype;    /* jd_dtype_t: storage type of W, H and w_judge */
+  int32_t device;   /* CUDA device ordinal the handle lives on */
+} jd_config_t;
+
+typedef struct jd_handle_s* jd_handle_t;
+
+typedef struct {
+  int32_t B;                   /* sequences in this call, 1..max_B */
+  int32_t M;                   /* draft tokens per sequence, 1..max_M */
+  const void* H;               /* [B, M+1, d] embeddings, dtype of the handle, 16-byte aligned */
+  const int32_t* draft_tokens; /* [B, M] drafted token ids x_j in [0, V) */
+  const float* draft_logits;   /* [B, M, V] draft-model logits; q_j = softmax at temperature 1 */
+  float tau;                   /* judge threshold in [0, 1]; accept iff score > tau (strict) */
+  uint64_t seed;               /* Philox key */
+  int32_t mode;                /* jd_mode_t */
+  int32_t resample;            /* jd_resample_t */
+  int32_t variant;             /* jd_variant_t; JD_VARIANT_AUTO in production */
+  /* outputs, always written */
+  int32_t* accept_len;         /* [B] number of accepted draft tokens, 0..M */
+  int32_t* next_token;         /* [B] the corrected (accept_len < M) or bonus (== M) token */
+  float* judge_scores;         /* [B, M] sigmoid(w . H[b,j+1] + b0) */
+  float* p_draft;              /* [B, M] p_j[x_j] */
+  /* optional outputs, may be NULL */
+  float* q_draft;              /* [B, M] q_j[x_j] */
+  uint8_t* masks;              /* [B, M] bit0 = standard test passed, bit1 = judge test passed */
+  float* row_max;              /* [B, M+1] max_v L[b,j,v] */
+  float* row_lse;              /* [B, M+1] log sum_v exp L[b,j,v] */
+  float* logits_debug;         /* [B, M+1, V] the logits; tests only, SIMT variant only */
+} jd_verify_args_t;
+
+/* Library version, major*10000 + minor*100 + patch. */
+int jd_version(void);
+
+/* Static text for a status code; never NULL. */
+const char* jd_status_string(jd_status_t s);
+
+/* Bytes of device workspace a handle with this configuration allocates (informational;
+ * the handle owns its workspace). Returns 0 for an invalid configuration. */
+size_t jd_workspace_bytes(const jd_config_t* cfg);
+
+/* Creates a handle on cfg->device: checks the architecture (JD_ERR_ARCH unless compute
+ * capability 10.x), allocates the workspace (JD_ERR_ALLOC) and stores the configuration.
+ * *out is set only on JD_OK. Not thread-safe per handle; distinct handles are independent. */
+jd_status_t jd_create(jd_handle_t* out, const jd_config_t* cfg);
+
+/* Frees the workspace. Synchronises the device first. NULL is accepted. */
+jd_status_t jd_destroy(jd_handle_t h);
+
+/* Registers the LM head W [V, d] and the judge head (w_judge [d], bias b_judge); device
+ * pointers in the handle's dtype, 16-byte aligned, borrowed until replaced or jd_destroy.
+ * The judge head is the paper's linear map R^d -> R (Sec. 4.1 "Model design and training",
+ * App. B.1). Builds the TMA descriptors of W. Must precede jd_verify. */
+jd_status_t jd_set_head(jd_handle_t h, const void* W, const void* w_judge, float b_judge);
+
+/* One verification call (steps 1-5 above) enqueued on `cuda_stream` (a cudaStream_t, NULL =
+ * default stream). Host-side checks return JD_ERR_INVALID_ARG / JD_ERR_UNSUPPORTED before
+ * anything is launched. Device-side conditions (clamped tokens, timed-out waits) are recorded
+ * in the handle's device status word, read with jd_last_device_status. Calls on one handle
+ * must be ordered on the device (same stream or explicit dependencies): they share the
+ * workspace. */
+jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* args, void* cuda_stream);
+
+/* Same call for callers whose per-step data live in HOST memory: `args` holds HOST pointers
+ * for H, draft_tokens, draft_logits and for every output (pinned memory recommended; W stays
+ * on the device via jd_set_head). Inputs are copied to handle-owned device staging buffers,
+ * the verification runs, the outputs are copied back, and the stream is synchronised before
+ * returning. logits_debug must be NULL. */
+jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* args, void* cuda_stream);
+
+/* Synchronises the stream of the handle's last jd_verify and copies the device status word:
+ * *out = JD_OK, JD_ERR_TIMEOUT or JD_ERR_BAD_TOKEN. */
+jd_status_t jd_last_device_status(jd_handle_t h, int* out);
+
+/* Variant the last jd_verify on this handle ran (jd_variant_t), 0 before the first call, and
+ * the number of kernels it launched. Either pointer may be NULL. */
+jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launches);
+
+/* Test helper: fills out[i] = Philox uniform for (seed, b[i], slot[i], stream[i]), i < n, with
+ * the device generator; device pointers. Used to compare the generator bit for bit with an
+ * independent host implementation. */
+jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot,
+                               const int32_t* stream, int32_t n, float* out, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JD_H_ */

@@ -1,0 +1,349 @@
+// C-ABI layer: handle, argument validation, variant choice, host-buffer entry point.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "jd_kernels.h"
+
+using namespace jd;
+
+struct jd_handle_s {
+  jd_config_t cfg;
+  int num_sms;
+  void* ws_base;
+  size_t ws_bytes;
+  Workspace ws;
+  const void* W;
+  const void* w_judge;
+  float b_judge;
+  bool head_set;
+  bool tm_w_ok;
+  CUtensorMap tm_w;        // W as a [V, d] bf16 tensor, box 64 x 128, 128-byte swizzle
+  cudaStream_t last_stream;
+  int last_variant;
+  int last_launches;
+  // device staging of the host-buffer entry point (allocated on first use)
+  void* st_H;
+  int32_t* st_x;
+  float* st_dl;
+  void* st_out;            // accept_len | next_token | judge_scores | p_draft | q_draft | row_max | row_lse | masks
+  size_t st_out_bytes;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// bf16 [rows, d] row-major tensor, box = 64 columns (128 bytes) x box_rows, 128-byte swizzle,
+// out-of-range rows read as zero.
+bool make_tensor_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t d, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {d, rows};
+  const cuuint64_t strides[1] = {d * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool config_ok(const jd_config_t* c) {
+  if (!c) return false;
+  if (c->max_B < 1 || c->max_M < 1 || c->d < 1 || c->V < 2) return false;
+  if (c->dtype != JD_DTYPE_F32 && c->dtype != JD_DTYPE_BF16) return false;
+  if ((int64_t)c->max_B * (c->max_M + 1) > (1 << 20)) return false;
+  return true;
+}
+
+// Carves the workspace; with base == nullptr only measures it.
+size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
+  const size_t maxB = c.max_B, maxR = (size_t)c.max_B * (c.max_M + 1), maxBM = (size_t)c.max_B * c.max_M;
+  const size_t np = std::max<size_t>((c.V + kVocabTile - 1) / kVocabTile, kMaxCtas);
+  const size_t nq = std::max<size_t>((c.V + 8191) / 8192, kMaxCtas);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    char* p = base ? base + off : nullptr;
+    off += align_up(bytes, 256);
+    return p;
+  };
+  Workspace w;
+  w.part_max = (float*)take(maxR * np * 4);
+  w.part_sum = (float*)take(maxR * np * 4);
+  w.gath = (float*)take(maxR * 4);
+  w.qpart_max = (float*)take(maxBM * nq * 4);
+  w.qpart_sum = (float*)take(maxBM * nq * 4);
+  w.qgath = (float*)take(maxBM * 4);
+  w.judge_logit = (float*)take(maxBM * 4);
+  w.row_max = (float*)take(maxR * 4);
+  w.row_lse = (float*)take(maxR * 4);
+  w.q_lse = (float*)take(maxBM * 4);
+  w.sel_row = (int*)take(maxB * 4);
+  w.sel_kind = (int*)take(maxB * 4);
+  w.sel_lse_p = (float*)take(maxB * 4);
+  w.sel_lse_q = (float*)take(maxB * 4);
+  w.sel_u = (float*)take(maxB * 4);
+  w.mass_r = (double*)take(maxB * np * 8);
+  w.mass_p = (double*)take(maxB * np * 8);
+  w.w_sel = (float*)take(maxB * (size_t)c.V * 4);
+  w.p_sel = (float*)take(maxB * (size_t)c.V * 4);
+  w.status = (unsigned*)take(256);
+  w.barrier = (unsigned*)take(256);
+  w.np_cap = (int)np;
+  w.nq_cap = (int)nq;
+  if (ws) *ws = w;
+  return off;
+}
+
+size_t elem_size(int dtype) { return dtype == JD_DTYPE_BF16 ? 2 : 4; }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+jd_status_t validate(jd_handle_t h, const jd_verify_args_t* a) {
+  if (!h || !a) return JD_ERR_INVALID_ARG;
+  if (!h->head_set) return JD_ERR_INVALID_ARG;
+  if (a->B < 1 || a->B > h->cfg.max_B || a->M < 1 || a->M > h->cfg.max_M) return JD_ERR_INVALID_ARG;
+  if (!a->H || !a->draft_tokens || !a->draft_logits) return JD_ERR_INVALID_ARG;
+  if (!a->accept_len || !a->next_token || !a->judge_scores || !a->p_draft) return JD_ERR_INVALID_ARG;
+  if (!(a->tau >= 0.f && a->tau <= 1.f)) return JD_ERR_INVALID_ARG;
+  if (a->mode < JD_MODE_STANDARD || a->mode > JD_MODE_JUDGE_OR_STANDARD) return JD_ERR_INVALID_ARG;
+  if (a->resample < JD_RESAMPLE_RESIDUAL || a->resample > JD_RESAMPLE_TARGET_P) return JD_ERR_INVALID_ARG;
+  if (a->variant < JD_VARIANT_AUTO || a->variant > JD_VARIANT_BATCHED) return JD_ERR_INVALID_ARG;
+  return JD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int jd_version(void) { return 100; }
+
+const char* jd_status_string(jd_status_t s) {
+  switch (s) {
+    case JD_OK: return "ok";
+    case JD_ERR_INVALID_ARG: return "invalid argument";
+    case JD_ERR_UNSUPPORTED: return "unsupported shape or dtype for the requested variant";
+    case JD_ERR_ARCH: return "device is not compute capability 10.x";
+    case JD_ERR_ALLOC: return "allocation failed";
+    case JD_ERR_CUDA: return "CUDA call failed";
+    case JD_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case JD_ERR_BAD_TOKEN: return "a draft token was outside the vocabulary and was clamped";
+  }
+  return "unknown status";
+}
+
+size_t jd_workspace_bytes(const jd_config_t* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return carve(*cfg, nullptr, nullptr);
+}
+
+jd_status_t jd_create(jd_handle_t* out, const jd_config_t* cfg) {
+  if (!out || !config_ok(cfg)) return JD_ERR_INVALID_ARG;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) return JD_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return JD_ERR_CUDA;
+  if (prop.major != 10) return JD_ERR_ARCH;
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return JD_ERR_CUDA;
+  jd_handle_s* h = new (std::nothrow) jd_handle_s();
+  if (!h) return JD_ERR_ALLOC;
+  std::memset(h, 0, sizeof(*h));
+  h->cfg = *cfg;
+  h->num_sms = prop.multiProcessorCount;
+  h->ws_bytes = carve(*cfg, nullptr, nullptr);
+  if (cudaMalloc(&h->ws_base, h->ws_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    delete h;
+    return JD_ERR_ALLOC;
+  }
+  carve(*cfg, (char*)h->ws_base, &h->ws);
+  if (cudaMemset(h->ws_base, 0, h->ws_bytes) != cudaSuccess) {
+    cudaFree(h->ws_base);
+    delete h;
+    return JD_ERR_CUDA;
+  }
+  *out = h;
+  return JD_OK;
+}
+
+jd_status_t jd_destroy(jd_handle_t h) {
+  if (!h) return JD_OK;
+  cudaSetDevice(h->cfg.device);
+  cudaDeviceSynchronize();
+  cudaFree(h->ws_base);
+  cudaFree(h->st_H);
+  cudaFree(h->st_x);
+  cudaFree(h->st_dl);
+  cudaFree(h->st_out);
+  delete h;
+  return JD_OK;
+}
+
+jd_status_t jd_set_head(jd_handle_t h, const void* W, const void* w_judge, float b_judge) {
+  if (!h || !W || !w_judge) return JD_ERR_INVALID_ARG;
+  if (!aligned16(W) || !aligned16(w_judge)) return JD_ERR_INVALID_ARG;
+  h->W = W;
+  h->w_judge = w_judge;
+  h->b_judge = b_judge;
+  h->head_set = true;
+  h->tm_w_ok = false;
+  if (h->cfg.dtype == JD_DTYPE_BF16 && h->cfg.d % 64 == 0)
+    h->tm_w_ok = make_tensor_map(&h->tm_w, W, (uint64_t)h->cfg.V, (uint64_t)h->cfg.d, 128);
+  return JD_OK;
+}
+
+jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_stream) {
+  jd_status_t v = validate(h, a);
+  if (v != JD_OK) return v;
+  if (!aligned16(a->H)) return JD_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const jd_config_t& c = h->cfg;
+  const int R = a->B * (a->M + 1);
+
+  CallParams cp;
+  cp.B = a->B; cp.M = a->M; cp.d = c.d; cp.V = c.V;
+  cp.draft_tokens = a->draft_tokens;
+  cp.draft_logits = a->draft_logits;
+  cp.tau = a->tau; cp.b_judge = h->b_judge; cp.seed = a->seed;
+  cp.mode = a->mode; cp.resample = a->resample;
+  cp.accept_len = a->accept_len; cp.next_token = a->next_token;
+  cp.judge_scores = a->judge_scores; cp.p_draft = a->p_draft;
+  cp.q_draft = a->q_draft; cp.masks = a->masks;
+  cp.row_max_out = a->row_max; cp.row_lse_out = a->row_lse;
+
+  FusedPlan plan;
+  const bool fused_ok = h->tm_w_ok && fused_supported(c.dtype, R, c.d, c.V, h->num_sms, &plan);
+  int variant = a->variant;
+  if (variant == JD_VARIANT_AUTO) variant = (fused_ok && !a->logits_debug) ? JD_VARIANT_FUSED : JD_VARIANT_SIMT;
+  if (variant == JD_VARIANT_FUSED && (!fused_ok || a->logits_debug)) return JD_ERR_UNSUPPORTED;
+  if (variant == JD_VARIANT_BATCHED) return JD_ERR_UNSUPPORTED;
+
+  if (cudaSetDevice(c.device) != cudaSuccess) return JD_ERR_CUDA;
+  if (cudaMemsetAsync(h->ws.status, 0, sizeof(unsigned), st) != cudaSuccess) return JD_ERR_CUDA;
+  int launches = 0;
+  if (variant == JD_VARIANT_SIMT) {
+    launches = run_simt(cp, h->ws, h->W, h->w_judge, a->H, c.dtype, a->logits_debug, st);
+  } else {
+    CUtensorMap tm_h;
+    if (!make_tensor_map(&tm_h, a->H, (uint64_t)R, (uint64_t)c.d, (uint32_t)plan.n_pad)) return JD_ERR_CUDA;
+    cudaError_t err = cudaSuccess;
+    launches = run_fused(cp, h->ws, h->tm_w, tm_h, a->H, h->w_judge, plan, st, &err);
+    if (launches < 0) return JD_ERR_CUDA;
+  }
+  if (cudaGetLastError() != cudaSuccess) return JD_ERR_CUDA;
+  h->last_stream = st;
+  h->last_variant = variant;
+  h->last_launches = launches;
+  return JD_OK;
+}
+
+jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* a, void* cuda_stream) {
+  jd_status_t v = validate(h, a);
+  if (v != JD_OK) return v;
+  if (a->logits_debug) return JD_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const jd_config_t& c = h->cfg;
+  if (cudaSetDevice(c.device) != cudaSuccess) return JD_ERR_CUDA;
+  const size_t maxB = c.max_B, maxR = (size_t)c.max_B * (c.max_M + 1), maxBM = (size_t)c.max_B * c.max_M;
+  if (!h->st_H) {
+    h->st_out_bytes = align_up(maxB * 4, 256) * 2 + align_up(maxBM * 4, 256) * 3 + align_up(maxR * 4, 256) * 2 +
+                      align_up(maxBM, 256);
+    if (cudaMalloc(&h->st_H, maxR * c.d * elem_size(c.dtype)) != cudaSuccess ||
+        cudaMalloc((void**)&h->st_x, maxBM * 4) != cudaSuccess ||
+        cudaMalloc((void**)&h->st_dl, maxBM * (size_t)c.V * 4) != cudaSuccess ||
+        cudaMalloc(&h->st_out, h->st_out_bytes) != cudaSuccess) {
+      cudaGetLastError();
+      cudaFree(h->st_H); cudaFree(h->st_x); cudaFree(h->st_dl); cudaFree(h->st_out);
+      h->st_H = nullptr; h->st_x = nullptr; h->st_dl = nullptr; h->st_out = nullptr;
+      return JD_ERR_ALLOC;
+    }
+  }
+  const size_t B = a->B, R = (size_t)a->B * (a->M + 1), BM = (size_t)a->B * a->M;
+  char* o = (char*)h->st_out;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { char* p = o + off; off += align_up(bytes, 256); return p; };
+  int32_t* d_acc = (int32_t*)take(maxB * 4);
+  int32_t* d_next = (int32_t*)take(maxB * 4);
+  float* d_js = (float*)take(maxBM * 4);
+  float* d_pd = (float*)take(maxBM * 4);
+  float* d_qd = (float*)take(maxBM * 4);
+  float* d_rm = (float*)take(maxR * 4);
+  float* d_rl = (float*)take(maxR * 4);
+  uint8_t* d_mk = (uint8_t*)take(maxBM);
+
+  if (cudaMemcpyAsync(h->st_H, a->H, R * c.d * elem_size(c.dtype), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(h->st_x, a->draft_tokens, BM * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(h->st_dl, a->draft_logits, BM * (size_t)c.V * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return JD_ERR_CUDA;
+
+  jd_verify_args_t dev = *a;
+  dev.H = h->st_H; dev.draft_tokens = h->st_x; dev.draft_logits = h->st_dl;
+  dev.accept_len = d_acc; dev.next_token = d_next; dev.judge_scores = d_js; dev.p_draft = d_pd;
+  dev.q_draft = a->q_draft ? d_qd : nullptr;
+  dev.masks = a->masks ? d_mk : nullptr;
+  dev.row_max = a->row_max ? d_rm : nullptr;
+  dev.row_lse = a->row_lse ? d_rl : nullptr;
+  jd_status_t s = jd_verify(h, &dev, cuda_stream);
+  if (s != JD_OK) return s;
+
+  bool ok = cudaMemcpyAsync(a->accept_len, d_acc, B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+            cudaMemcpyAsync(a->next_token, d_next, B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+            cudaMemcpyAsync(a->judge_scores, d_js, BM * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
+            cudaMemcpyAsync(a->p_draft, d_pd, BM * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (ok && a->q_draft) ok = cudaMemcpyAsync(a->q_draft, d_qd, BM * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (ok && a->masks) ok = cudaMemcpyAsync(a->masks, d_mk, BM, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (ok && a->row_max) ok = cudaMemcpyAsync(a->row_max, d_rm, R * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (ok && a->row_lse) ok = cudaMemcpyAsync(a->row_lse, d_rl, R * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (!ok) return JD_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return JD_ERR_CUDA;
+  return JD_OK;
+}
+
+jd_status_t jd_last_device_status(jd_handle_t h, int* out) {
+  if (!h || !out) return JD_ERR_INVALID_ARG;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return JD_ERR_CUDA;
+  if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return JD_ERR_CUDA;
+  unsigned s = 0;
+  if (cudaMemcpy(&s, h->ws.status, sizeof(s), cudaMemcpyDeviceToHost) != cudaSuccess) return JD_ERR_CUDA;
+  *out = (int)s;
+  return JD_OK;
+}
+
+jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launches) {
+  if (!h) return JD_ERR_INVALID_ARG;
+  if (variant) *variant = h->last_variant;
+  if (kernel_launches) *kernel_launches = h->last_launches;
+  return JD_OK;
+}
+
+jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot, const int32_t* stream,
+                               int32_t n, float* out, void* cuda_stream) {
+  if (!b || !slot || !stream || !out || n < 0) return JD_ERR_INVALID_ARG;
+  if (n == 0) return JD_OK;
+  launch_philox_uniforms(seed, b, slot, stream, n, out, (cudaStream_t)cuda_stream);
+  return cudaGetLastError() == cudaSuccess ? JD_OK : JD_ERR_CUDA;
+}
+
+}  // extern "C"

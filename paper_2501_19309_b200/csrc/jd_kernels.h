@@ -1,0 +1,34 @@
+// Internal interface between the C-ABI layer and the kernel families.
+#pragma once
+
+#include <cuda.h>
+
+#include "jd_common.cuh"
+
+namespace jd {
+
+// CUDA-core pipeline (jd_simt.cu). Each returns after enqueueing on `st`.
+int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const void* w_judge, const void* H, int dtype,
+             float* logits_debug, cudaStream_t st);
+int launch_q_stats(const CallParams& cp, const Workspace& ws, cudaStream_t st);   // returns partials per draft row
+void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, const void* w, int dtype, cudaStream_t st);
+void launch_decide(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st);
+void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream_t st);
+void launch_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot, const int32_t* stream, int n,
+                            float* out, cudaStream_t st);
+
+// Persistent tensor-core kernel with the logits parked in tensor memory (jd_fused_sm100.cu).
+struct FusedPlan {
+  int num_ctas;       // persistent grid = number of SMs
+  int n_pad;          // MMA N: rows padded to a multiple of 16
+  int max_tiles;      // vocabulary tiles of the busiest CTA
+  int tmem_tiles;     // tiles whose accumulators stay in tensor memory
+  size_t smem_bytes;  // dynamic shared memory of the launch
+  int stages;         // W ring depth
+};
+bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan);
+// Returns the number of kernels launched, or -1 with *err set.
+int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
+              const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err);
+
+}  // namespace jd

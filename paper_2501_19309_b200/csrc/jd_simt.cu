@@ -1,0 +1,320 @@
+// CUDA-core pipeline of the verification step: any shape, f32 or bf16 storage, fp32
+// arithmetic. It is the variant for shapes the tensor-core kernels do not cover (fp32
+// heads, ragged d) and the on-device second opinion the tests compare the fused kernels
+// with. Its stages that do not touch W (draft statistics, judge dot products, decision,
+// token location) are shared with the batched tensor-core variant.
+#include "jd_kernels.h"
+
+namespace jd {
+
+// -----------------------------------------------------------------------------------------
+// Stage 1: logits of a [128 vocab] x [16 rows] tile by smem-tiled FMA.
+//   kSample == false: per-(row, vocab tile) softmax partials + gather of L[row, x_j]
+//   kSample == true : rows are the selected rows (one per sequence); writes the sampling
+//                     weights and p of that row plus their per-tile masses
+// -----------------------------------------------------------------------------------------
+constexpr int kSimtRows = 16;
+constexpr int kSimtK = 32;
+
+template <typename T, bool kSample>
+__global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, Workspace ws, const T* __restrict__ W,
+                                                                 const T* __restrict__ H, int R, int np,
+                                                                 float* __restrict__ logits_debug) {
+  __shared__ float sW[kVocabTile][kSimtK + 1];
+  __shared__ __align__(16) float sH[kSimtRows][kSimtK];
+  __shared__ float s_m[4][kSimtRows], s_s[4][kSimtRows];
+  __shared__ double s_d[2][4][kSimtRows];
+  __shared__ int s_row[kSimtRows];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tile = blockIdx.x;
+  const int v = tile * kVocabTile + tid;
+  const int r0 = blockIdx.y * kSimtRows;
+  const int d = cp.d, V = cp.V;
+
+  if (tid < kSimtRows) {
+    const int r = r0 + tid;
+    s_row[tid] = (r < R) ? (kSample ? ws.sel_row[r] : r) : -1;
+  }
+  __syncthreads();
+
+  float acc[kSimtRows];
+#pragma unroll
+  for (int i = 0; i < kSimtRows; ++i) acc[i] = 0.f;
+
+  for (int k0 = 0; k0 < d; k0 += kSimtK) {
+    // W tile: 128 rows x 32 k, coalesced along k
+    for (int i = tid; i < kVocabTile * kSimtK; i += kVocabTile) {
+      const int rr = i / kSimtK, kk = i % kSimtK;
+      const int vv = tile * kVocabTile + rr;
+      sW[rr][kk] = (vv < V && k0 + kk < d) ? to_float<T>(W[(size_t)vv * d + k0 + kk]) : 0.f;
+    }
+    for (int i = tid; i < kSimtRows * kSimtK; i += kVocabTile) {
+      const int rr = i / kSimtK, kk = i % kSimtK;
+      const int row = s_row[rr];
+      sH[rr][kk] = (row >= 0 && k0 + kk < d) ? to_float<T>(H[(size_t)row * d + k0 + kk]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kSimtK; kk += 4) {
+      const float w0 = sW[tid][kk], w1 = sW[tid][kk + 1], w2 = sW[tid][kk + 2], w3 = sW[tid][kk + 3];
+#pragma unroll
+      for (int i = 0; i < kSimtRows; ++i) {
+        const float4 h = *reinterpret_cast<const float4*>(&sH[i][kk]);
+        acc[i] = fmaf(w0, h.x, acc[i]);
+        acc[i] = fmaf(w1, h.y, acc[i]);
+        acc[i] = fmaf(w2, h.z, acc[i]);
+        acc[i] = fmaf(w3, h.w, acc[i]);
+      }
+    }
+    __syncthreads();
+  }
+
+  const bool valid_v = v < V;
+  if (!kSample) {
+#pragma unroll
+    for (int i = 0; i < kSimtRows; ++i) {
+      const int row = s_row[i];
+      float m = (valid_v && row >= 0) ? acc[i] : -INFINITY;
+      float s = (valid_v && row >= 0) ? 1.f : 0.f;
+      ms_warp_reduce(m, s);
+      if (lane == 0) { s_m[warp][i] = m; s_s[warp][i] = s; }
+      if (row >= 0 && valid_v) {
+        if (logits_debug) logits_debug[(size_t)row * V + v] = acc[i];
+        const int b = row / (cp.M + 1), j = row % (cp.M + 1);
+        if (j < cp.M) {
+          int x = cp.draft_tokens[b * cp.M + j];
+          if (x < 0 || x >= V) { set_status(ws.status, JD_ERR_BAD_TOKEN); x = min(max(x, 0), V - 1); }
+          if (x == v) ws.gath[row] = acc[i];
+        }
+      }
+    }
+    __syncthreads();
+    if (tid < kSimtRows && s_row[tid] >= 0) {
+      float m = s_m[0][tid], s = s_s[0][tid];
+      for (int w = 1; w < 4; ++w) ms_combine(m, s, s_m[w][tid], s_s[w][tid]);
+      ws.part_max[(size_t)s_row[tid] * np + tile] = m;
+      ws.part_sum[(size_t)s_row[tid] * np + tile] = s;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < kSimtRows; ++i) {
+      const int row = s_row[i];
+      const int b = r0 + i;
+      float p = 0.f, r = 0.f;
+      if (row >= 0 && valid_v) {
+        const int kind = ws.sel_kind[b];
+        const int a = row % (cp.M + 1);
+        const float dlv = (kind == 0) ? cp.draft_logits[((size_t)b * cp.M + a) * V + v] : 0.f;
+        sample_weights(acc[i], ws.sel_lse_p[b], kind, dlv, ws.sel_lse_q[b], p, r);
+        ws.w_sel[(size_t)b * V + v] = r;
+        ws.p_sel[(size_t)b * V + v] = p;
+      }
+      const double dr = warp_sum_double((double)r), dp = warp_sum_double((double)p);
+      if (lane == 0) { s_d[0][warp][i] = dr; s_d[1][warp][i] = dp; }
+    }
+    __syncthreads();
+    if (tid < kSimtRows && s_row[tid] >= 0) {
+      const int b = r0 + tid;
+      ws.mass_r[(size_t)b * np + tile] = (s_d[0][0][tid] + s_d[0][1][tid]) + (s_d[0][2][tid] + s_d[0][3][tid]);
+      ws.mass_p[(size_t)b * np + tile] = (s_d[1][0][tid] + s_d[1][1][tid]) + (s_d[1][2][tid] + s_d[1][3][tid]);
+    }
+  }
+}
+
+// -----------------------------------------------------------------------------------------
+// Draft-row statistics: per (draft row, chunk) online (max, sum exp) and the gather of the
+// drafted token's logit. One block per chunk of kQChunk logits.
+// -----------------------------------------------------------------------------------------
+constexpr int kQChunk = 8192;
+
+__global__ void __launch_bounds__(256) q_stats_kernel(CallParams cp, Workspace ws, int nq) {
+  __shared__ float s_m[8], s_s[8];
+  const int bm = blockIdx.y, chunk = blockIdx.x;
+  const int V = cp.V;
+  const float* row = cp.draft_logits + (size_t)bm * V;
+  const int lo = chunk * kQChunk, hi = min(V, lo + kQChunk);
+  float m = -INFINITY, s = 0.f;
+  for (int v = lo + threadIdx.x; v < hi; v += blockDim.x) {
+    const float xv = row[v];
+    if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
+    else if (xv != -INFINITY) s += __expf(xv - m);
+  }
+  ms_warp_reduce(m, s);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) { s_m[warp] = m; s_s[warp] = s; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) ms_combine(m, s, s_m[w], s_s[w]);
+    ws.qpart_max[(size_t)bm * nq + chunk] = m;
+    ws.qpart_sum[(size_t)bm * nq + chunk] = s;
+    if (chunk == 0) {
+      int x = cp.draft_tokens[bm];
+      if (x < 0 || x >= V) { set_status(ws.status, JD_ERR_BAD_TOKEN); x = min(max(x, 0), V - 1); }
+      ws.qgath[bm] = row[x];
+    }
+  }
+}
+
+// Judge dot products: one block per draft slot, w . H[b, j+1].
+template <typename T>
+__global__ void __launch_bounds__(256) judge_dot_kernel(CallParams cp, Workspace ws, const T* __restrict__ H,
+                                                        const T* __restrict__ w) {
+  __shared__ float s_p[8];
+  const int bm = blockIdx.x;
+  const int b = bm / cp.M, j = bm % cp.M;
+  const T* h = H + ((size_t)b * (cp.M + 1) + j + 1) * cp.d;
+  float acc = 0.f;
+  for (int k = threadIdx.x; k < cp.d; k += blockDim.x) acc = fmaf(to_float<T>(w[k]), to_float<T>(h[k]), acc);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) s_p[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < 8; ++i) t += s_p[i];
+    ws.judge_logit[bm] = t;
+  }
+}
+
+// -----------------------------------------------------------------------------------------
+// Decision: one block per sequence. Warps first fold the partial statistics of the rows
+// (fixed order, so results repeat bit for bit), then warp 0 runs the tests.
+// -----------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) decide_kernel(CallParams cp, Workspace ws, int np, int nq) {
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int M = cp.M;
+  for (int j = warp; j <= M; j += 4) {
+    const int row = b * (M + 1) + j;
+    float m = -INFINITY, s = 0.f;
+    for (int i = lane; i < np; i += 32)
+      ms_combine(m, s, ws.part_max[(size_t)row * np + i], ws.part_sum[(size_t)row * np + i]);
+    ms_warp_reduce(m, s);
+    if (lane == 0) {
+      const float lse = m + logf(s);
+      ws.row_max[row] = m;
+      ws.row_lse[row] = lse;
+      if (cp.row_max_out) cp.row_max_out[row] = m;
+      if (cp.row_lse_out) cp.row_lse_out[row] = lse;
+    }
+  }
+  for (int j = warp; j < M; j += 4) {
+    const int bm = b * M + j;
+    float m = -INFINITY, s = 0.f;
+    for (int i = lane; i < nq; i += 32)
+      ms_combine(m, s, ws.qpart_max[(size_t)bm * nq + i], ws.qpart_sum[(size_t)bm * nq + i]);
+    ms_warp_reduce(m, s);
+    if (lane == 0) ws.q_lse[bm] = m + logf(s);
+  }
+  __syncthreads();
+  if (warp == 0) decide_sequence(cp, ws, b, true);
+}
+
+// -----------------------------------------------------------------------------------------
+// Token location: inverse CDF in ascending token id over the stored weights of the selected
+// row. Tile masses are prefix-summed in double; inside the owning tile the weights are added
+// one by one in double.
+// -----------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) locate_kernel(CallParams cp, Workspace ws, int np) {
+  const int b = blockIdx.x;
+  if (threadIdx.x != 0) return;
+  const int V = cp.V;
+  const int ntiles = (V + kVocabTile - 1) / kVocabTile;
+  const double* mass = ws.mass_r + (size_t)b * np;
+  const float* wv = ws.w_sel + (size_t)b * V;
+  double total = 0.0;
+  for (int t = 0; t < ntiles; ++t) total += mass[t];
+  if (!(total > 0.0)) {  // identically zero residual: draw from p
+    mass = ws.mass_p + (size_t)b * np;
+    wv = ws.p_sel + (size_t)b * V;
+    total = 0.0;
+    for (int t = 0; t < ntiles; ++t) total += mass[t];
+  }
+  const double T = (double)ws.sel_u[b] * total;
+  double prefix = 0.0;
+  int token = -1;
+  for (int t = 0; t < ntiles && token < 0; ++t) {
+    const double incl = prefix + mass[t];
+    if (incl > T) {
+      double c = prefix;
+      const int lo = t * kVocabTile, hi = min(V, lo + kVocabTile);
+      int last_pos = -1;
+      for (int vv = lo; vv < hi; ++vv) {
+        const float x = wv[vv];
+        c += (double)x;
+        if (x > 0.f) last_pos = vv;
+        if (c > T) { token = vv; break; }
+      }
+      if (token < 0) token = last_pos;  // summation-order rounding inside the tile
+    }
+    prefix = incl;
+  }
+  if (token < 0) {  // T >= total after rounding: the last token that carries mass
+    for (int vv = V - 1; vv >= 0; --vv)
+      if (wv[vv] > 0.f) { token = vv; break; }
+  }
+  cp.next_token[b] = token < 0 ? 0 : token;
+}
+
+__global__ void philox_uniforms_kernel(uint64_t seed, const int32_t* b, const int32_t* slot, const int32_t* stream,
+                                       int n, float* out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = philox_uniform(seed, b[i], slot[i], stream[i]);
+}
+
+// -----------------------------------------------------------------------------------------
+// host-side launchers
+// -----------------------------------------------------------------------------------------
+int launch_q_stats(const CallParams& cp, const Workspace& ws, cudaStream_t st) {
+  const int nq = (cp.V + kQChunk - 1) / kQChunk;
+  q_stats_kernel<<<dim3(nq, cp.B * cp.M), 256, 0, st>>>(cp, ws, nq);
+  return nq;
+}
+
+void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, const void* w, int dtype, cudaStream_t st) {
+  if (dtype == JD_DTYPE_BF16)
+    judge_dot_kernel<__nv_bfloat16><<<cp.B * cp.M, 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H, (const __nv_bfloat16*)w);
+  else
+    judge_dot_kernel<float><<<cp.B * cp.M, 256, 0, st>>>(cp, ws, (const float*)H, (const float*)w);
+}
+
+void launch_decide(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st) {
+  decide_kernel<<<cp.B, 128, 0, st>>>(cp, ws, np, nq);
+}
+
+void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream_t st) {
+  locate_kernel<<<cp.B, 32, 0, st>>>(cp, ws, np);
+}
+
+template <typename T>
+static void simt_logits(const CallParams& cp, const Workspace& ws, const void* W, const void* H, bool sample, int np,
+                        float* logits_debug, cudaStream_t st) {
+  const int R = sample ? cp.B : cp.B * (cp.M + 1);
+  dim3 grid(np, (R + kSimtRows - 1) / kSimtRows);
+  if (sample)
+    simt_logits_kernel<T, true><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, nullptr);
+  else
+    simt_logits_kernel<T, false><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, logits_debug);
+}
+
+int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const void* w_judge, const void* H, int dtype,
+             float* logits_debug, cudaStream_t st) {
+  const int np = (cp.V + kVocabTile - 1) / kVocabTile;
+  const int nq = launch_q_stats(cp, ws, st);
+  launch_judge(cp, ws, H, w_judge, dtype, st);
+  if (dtype == JD_DTYPE_BF16) simt_logits<__nv_bfloat16>(cp, ws, W, H, false, np, logits_debug, st);
+  else simt_logits<float>(cp, ws, W, H, false, np, logits_debug, st);
+  launch_decide(cp, ws, np, nq, st);
+  if (dtype == JD_DTYPE_BF16) simt_logits<__nv_bfloat16>(cp, ws, W, H, true, np, nullptr, st);
+  else simt_logits<float>(cp, ws, W, H, true, np, nullptr, st);
+  launch_locate(cp, ws, np, st);
+  return 6;
+}
+
+void launch_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot, const int32_t* stream, int n,
+                            float* out, cudaStream_t st) {
+  philox_uniforms_kernel<<<(n + 255) / 256, 256, 0, st>>>(seed, b, slot, stream, n, out);
+}
+
+}  // namespace jd

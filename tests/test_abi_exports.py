@@ -1,0 +1,46 @@
+"""The C-ABI library builds, loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+from paper_2501_19309_b200 import build as B
+from paper_2501_19309_b200 import jd
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    src = open(os.path.join(ROOT, "include", "jd.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    names = re.findall(r"\b(jd_[a-z_0-9]+)\s*\(", src)
+    return sorted(set(names))
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    path = B.build()
+    assert os.path.exists(path) and path == jd.library_path()
+    lib = ctypes.CDLL(path)
+    names = declared_functions()
+    assert set(jd.EXPORTS) <= set(names)
+    assert len(names) >= 11
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_calls_that_need_no_device():
+    assert jd.jd_version() >= 100
+    assert jd.jd_status_string(jd.JD_OK) == "ok"
+    assert "wait" in jd.jd_status_string(jd.JD_ERR_TIMEOUT)
+    cfg = jd.jd_config_t(4, 16, 8192, 128256, jd.JD_DTYPE_BF16, 0)
+    n = jd.jd_workspace_bytes(cfg)
+    assert 1 << 20 < n < 1 << 30
+    bad = jd.jd_config_t(0, 16, 8192, 128256, jd.JD_DTYPE_BF16, 0)
+    assert jd.jd_workspace_bytes(bad) == 0
+
+
+def test_struct_layout_matches_header_order():
+    src = open(os.path.join(ROOT, "include", "jd.h")).read()
+    body = src[src.index("typedef struct {\n  int32_t B;"):src.index("} jd_verify_args_t;")]
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    fields = re.findall(r"([A-Za-z_0-9]+)\s*;", body)
+    assert fields == [f[0] for f in jd.jd_verify_args_t._fields_]

@@ -1,0 +1,192 @@
+"""GPU parity: the library, called through its C ABI, against the CPU checker on the same
+seeded inputs.  Every test here needs a B200."""
+import numpy as np
+import pytest
+
+import jd_testlib as T
+from oracle import jd_oracle as O
+from paper_2501_19309_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+MODES = ("standard", "judge", "judge_or_standard")
+
+
+def run_case(wl, data_seed, modes=MODES, variant="auto", seeds=None, tau=None, check_logits=False,
+             sequences=None, expect_variant=None):
+    from paper_2501_19309_b200 import jd
+    inp = I.make_inputs(wl, data_seed)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    rep = T.Report()
+    for mode in modes:
+        for seed in (seeds or [inp.seed]):
+            out = ver.alloc_outputs(wl.B, wl.M, debug_logits=check_logits)
+            ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau if tau is None else tau, seed, mode,
+                       variant=variant, out=out)
+            assert ver.device_status() == jd.JD_OK
+            if expect_variant is not None:
+                assert ver.launch_info()[0] == jd.VARIANTS[expect_variant]
+            got = T.to_numpy(out)
+            ref = T.run_oracle(inp, mode, seed=seed, tau=tau, sequences=sequences, keep_logits=check_logits)
+            T.compare(got, ref, mode, wl.M, rep)
+            if check_logits:
+                T.compare_logits(got["logits_debug"], ref, rep)
+    ver.close()
+    return rep
+
+
+def test_philox_bit_equality_with_checker():
+    import torch
+    from paper_2501_19309_b200 import jd
+    n = 60000
+    rng = np.random.default_rng(0)
+    b = rng.integers(0, 1 << 20, n).astype(np.int32)
+    slot = rng.integers(0, 64, n).astype(np.int32)
+    stream = rng.integers(0, 2, n).astype(np.int32)
+    b[:4] = [0, 1, 2 ** 31 - 1, 5]
+    for seed in (0, 1, (0xDEADBEEF << 32) | 0x12345678):
+        tb, ts, tst = (torch.from_numpy(a).cuda() for a in (b, slot, stream))
+        out = torch.empty(n, dtype=torch.float32, device="cuda")
+        assert jd.jd_philox_uniforms(seed, tb.data_ptr(), ts.data_ptr(), tst.data_ptr(), n, out.data_ptr()) == 0
+        got = out.cpu().numpy().astype(np.float64)
+        m = n if seed == 0 else 3000
+        want = np.array([O.uniform24(seed, int(b[i]), int(slot[i]), int(stream[i])) for i in range(m)])
+        assert np.array_equal(got[:m], want)
+
+
+def test_cfg0_tiny_fp32_all_modes_with_logits():
+    rep = run_case(I.CONFIGS[0], 0, check_logits=True, expect_variant="simt")
+    assert rep.sequences == 3 and rep.max_rel_logit < 1e-4
+
+
+@pytest.mark.parametrize("B,M,d,V", [(1, 1, 64, 130), (2, 5, 192, 1037), (3, 33, 100, 515), (5, 8, 256, 4096 + 77)])
+def test_simt_bf16_ragged_shapes(B, M, d, V):
+    wl = I.CONFIGS[2].scaled("ragged", B=B, M=M, d=d, V=V)
+    rep = run_case(wl, 1, variant="simt", seeds=[0, 1, 2], check_logits=True)
+    assert rep.sequences == 9 * B
+
+
+def test_simt_fp32_ragged():
+    wl = I.CONFIGS[0].scaled("ragged32", B=2, M=3, d=77, V=333)
+    run_case(wl, 2, variant="simt", seeds=[0, 1], check_logits=True)
+
+
+def test_tau_extremes_and_literal_resampling():
+    from paper_2501_19309_b200 import jd
+    wl = I.CONFIGS[1].scaled("small", d=256, V=2048, B=3, M=6)
+    inp = I.make_inputs(wl, 5)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    res = {}
+    for tau in (0.0, 1.0):
+        for mode in MODES:
+            out = ver.verify(dev["H"], dev["x"], dev["dl"], tau, 3, mode)
+            got = T.to_numpy(out)
+            ref = T.run_oracle(inp, mode, seed=3, tau=tau)
+            T.compare(got, ref, mode, wl.M)
+            res[(tau, mode)] = got
+    # tau = 1: the judge never accepts, so the OR mode is the standard test (Sec. 4.1)
+    assert np.array_equal(res[(1.0, "judge_or_standard")]["accept_len"], res[(1.0, "standard")]["accept_len"])
+    assert np.array_equal(res[(1.0, "judge_or_standard")]["next_token"], res[(1.0, "standard")]["next_token"])
+    assert (res[(1.0, "judge")]["accept_len"] == 0).all()
+    assert (res[(0.0, "judge")]["accept_len"] == wl.M).all()          # sigmoid > 0 always
+    out = ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 3, "standard", resample="target_p")
+    ref = O.jd_oracle_verify(inp.W, inp.w_judge, inp.b_judge, inp.H, inp.draft_tokens, inp.draft_logits, 0.5, 3,
+                             "standard", "target_p")
+    T.compare(T.to_numpy(out), ref, "standard", wl.M)
+    ver.close()
+
+
+def test_or_mode_monotone_on_device():
+    wl = I.CONFIGS[2].scaled("small", d=128, V=1500, B=8, M=12)
+    inp = I.make_inputs(wl, 9)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    for seed in range(4):
+        a = {m: T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, seed, m))["accept_len"] for m in MODES}
+        assert (a["judge_or_standard"] >= np.maximum(a["standard"], a["judge"])).all()
+        assert (a["judge_or_standard"] <= wl.M).all() and (a["standard"] >= 0).all()
+    ver.close()
+
+
+def test_q_equals_p_accepts_everything():
+    import torch
+    wl = I.CONFIGS[1].scaled("small", d=128, V=1000, B=2, M=7)
+    inp = I.make_inputs(wl, 4)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    out = ver.alloc_outputs(wl.B, wl.M, debug_logits=True)
+    ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "standard", variant="simt", out=out)
+    dl = out["logits_debug"][:, :wl.M, :].contiguous()          # the device's own logits as draft logits
+    for seed in range(5):
+        got = T.to_numpy(ver.verify(dev["H"], dev["x"], dl, 0.5, seed, "standard", variant="simt"))
+        assert (got["accept_len"] == wl.M).all()
+        assert np.allclose(got["p_draft"], got["q_draft"], rtol=1e-5)
+    ver.close()
+
+
+def test_zero_draft_probability_and_bad_token_status():
+    import torch
+    from paper_2501_19309_b200 import jd
+    wl = I.CONFIGS[1].scaled("small", d=64, V=600, B=1, M=3)
+    inp = I.make_inputs(wl, 6)
+    inp.draft_logits[0, 0, inp.draft_tokens[0, 0]] = -np.inf
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    got = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "standard"))
+    ref = T.run_oracle(inp, "standard", seed=0)
+    T.compare(got, ref, "standard", wl.M)
+    assert got["q_draft"][0, 0] == 0.0 and got["masks"][0, 0] & 1
+    x_bad = dev["x"].clone()
+    x_bad[0, 1] = wl.V + 5
+    ver.verify(dev["H"], x_bad, dev["dl"], 0.5, 0, "standard")
+    assert ver.device_status() == jd.JD_ERR_BAD_TOKEN
+    ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "standard")
+    assert ver.device_status() == jd.JD_OK                   # the status word is per call
+    ver.close()
+
+
+def test_argument_validation_returns_codes():
+    import torch
+    from paper_2501_19309_b200 import jd
+    wl = I.CONFIGS[1].scaled("small", d=64, V=600, B=2, M=3)
+    inp = I.make_inputs(wl, 7)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    a, out = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0)
+    assert jd.jd_verify(ver.h, a) == jd.JD_OK
+    for field, value in (("B", 0), ("B", 3), ("M", 0), ("M", 4), ("tau", 1.5), ("tau", -0.1), ("mode", 3),
+                         ("resample", 2), ("variant", 9), ("H", None), ("draft_tokens", None),
+                         ("accept_len", None), ("p_draft", None)):
+        a2, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, out=out)
+        setattr(a2, field, value)
+        assert jd.jd_verify(ver.h, a2) == jd.JD_ERR_INVALID_ARG, field
+    a3, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, out=out)
+    a3.H = dev["H"].data_ptr() + 2                           # misaligned
+    assert jd.jd_verify(ver.h, a3) == jd.JD_ERR_INVALID_ARG
+    v2 = jd.Verifier(2, 3, wl.d, wl.V, "bf16")
+    a4, _ = v2.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, out=out)
+    assert jd.jd_verify(v2.h, a4) == jd.JD_ERR_INVALID_ARG   # no head registered yet
+    v2.close()
+    with pytest.raises(jd.JdError):
+        jd.jd_create(jd.jd_config_t(1, 1, 64, 600, 5, 0))
+    ver.close()
+
+
+def test_host_buffer_entry_point_matches_device_call_and_is_repeatable():
+    import torch
+    wl = I.CONFIGS[2].scaled("small", d=256, V=3000, B=4, M=9)
+    inp = I.make_inputs(wl, 8)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    d1 = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 11, "judge_or_standard"))
+    d2 = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 11, "judge_or_standard"))
+    hostH = torch.from_numpy(inp.H).view(torch.bfloat16).pin_memory()
+    hx = torch.from_numpy(inp.draft_tokens).pin_memory()
+    hdl = torch.from_numpy(inp.draft_logits).pin_memory()
+    h1 = {k: v.numpy().copy() for k, v in ver.verify_host(hostH, hx, hdl, 0.5, 11, "judge_or_standard").items()}
+    for k in d1:
+        assert np.array_equal(d1[k], d2[k]), k              # run-to-run determinism
+        assert np.array_equal(d1[k], h1[k]), k
+    ver.close()

@@ -241,7 +241,8 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   if (variant == JD_VARIANT_BATCHED) return JD_ERR_UNSUPPORTED;
 
   if (cudaSetDevice(c.device) != cudaSuccess) return JD_ERR_CUDA;
-  if (cudaMemsetAsync(h->ws.status, 0, sizeof(unsigned), st) != cudaSuccess) return JD_ERR_CUDA;
+  // status word and the grid-barrier counters behind it start every call at zero
+  if (cudaMemsetAsync(h->ws.status, 0, 512, st) != cudaSuccess) return JD_ERR_CUDA;
   int launches = 0;
   if (variant == JD_VARIANT_SIMT) {
     launches = run_simt(cp, h->ws, h->W, h->w_judge, a->H, c.dtype, a->logits_debug, st);

@@ -128,7 +128,9 @@ struct CallParams {
 // Decision step for one sequence b, executed by one warp (Eq. 4, Sec. 4.1 "Inference"):
 // given the rows' log-normalisers, the gathered logits and the judge logits, evaluates both
 // tests for every slot, combines them by mode, finds the accepted prefix and records which
-// row the next token is drawn from. Every lane returns the accepted length.
+// row the next token is drawn from. Every lane returns the accepted length. gath, qgath and
+// judge_logit are always global memory (possibly written by other CTAs of the same grid, hence
+// the L2 loads); the log-normalisers and the sel_* outputs may live in shared memory.
 __device__ __forceinline__ int decide_sequence(const CallParams& cp, const Workspace& ws, int b,
                                                bool write_outputs) {
   const int lane = threadIdx.x & 31;
@@ -140,11 +142,11 @@ __device__ __forceinline__ int decide_sequence(const CallParams& cp, const Works
     if (j < M) {
       const int row = b * (M + 1) + j;
       const int bm = b * M + j;
-      const float P = expf(ws.gath[row] - ws.row_lse[row]);
-      const float Q = expf(ws.qgath[bm] - ws.q_lse[bm]);
+      const float P = expf(__ldcg(ws.gath + row) - ws.row_lse[row]);
+      const float Q = expf(__ldcg(ws.qgath + bm) - ws.q_lse[bm]);
       const float u = philox_uniform(cp.seed, b, j, 0);
       const bool z_std = (u * Q < P);
-      const float s = 1.0f / (1.0f + expf(-(ws.judge_logit[bm] + cp.b_judge)));
+      const float s = 1.0f / (1.0f + expf(-(__ldcg(ws.judge_logit + bm) + cp.b_judge)));
       const bool z_judge = (s > cp.tau);
       ok = cp.mode == JD_MODE_STANDARD ? z_std : (cp.mode == JD_MODE_JUDGE ? z_judge : (z_std || z_judge));
       if (write_outputs) {

@@ -1,7 +1,743 @@
-// placeholder until the tensor-core kernel lands
+// Persistent tensor-core kernel for small row counts (B*(M+1) <= 96): one cooperative launch,
+// one CTA per SM, the whole verification step in a single kernel.
+//
+// Orientation ("swap-AB"): the MMA's M axis (128 TMEM lanes) is the vocabulary, its N axis
+// (TMEM columns) the rows of H. D[v, r] = sum_k W[v, k] H[r, k]. Each CTA owns a contiguous
+// range of 128-entry vocabulary tiles (at most seven for V = 128256 on 148 SMs) and keeps the
+// fp32 logits of ALL of them on chip until the call ends: tile i occupies TMEM columns
+// [i*N_PAD, (i+1)*N_PAD); tiles that do not fit in the 512 columns are computed first and moved
+// to shared memory. The logits never reach device memory.
+//
+// Warp roles (192 threads): warps 0-3 statistics / decisions / sampling (one TMEM lane
+// quadrant each), warp 4 lane 0 TMA producer, warp 5 lane 0 MMA issuer (warp 5 owns the TMEM
+// allocation).
+//
+// Main loop, K-outer: for every 64-wide slice of d the H slice [N_PAD x 64] is loaded once and
+// multiplied with the W slice [128 x 64] of every tile of the group, so W streams from HBM
+// exactly once and H is re-read (from L2) once per group, not once per tile.
+//
+// After the main loop the grid meets twice:
+//   per-CTA (max, sum exp) of every row, logit of the drafted tokens        -> barrier 1
+//   every CTA folds the statistics, runs the tests and the prefix rule (identical results),
+//   then computes its slice of the sampling mass of each sequence's selected row -> barrier 2
+//   the CTA whose slice contains T = u * total mass locates the token.
+// Both barriers are counters in global memory, legal because the launch is cooperative (all
+// CTAs co-resident); every wait in the kernel is bounded and reports JD_ERR_TIMEOUT.
+#include <cooperative_groups.h>
+
 #include "jd_kernels.h"
+
 namespace jd {
-bool fused_supported(int, int, int, int, int, FusedPlan*) { return false; }
-int run_fused(const CallParams&, const Workspace&, const CUtensorMap&, const CUtensorMap&, const void*, const void*,
-              const FusedPlan&, cudaStream_t, cudaError_t* err) { *err = cudaErrorNotSupported; return -1; }
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr int kBlockK = 64;                      // bf16 elements per k-slice = one 128-byte swizzle row
+constexpr int kWStageBytes = kVocabTile * 128;   // 16 KB
+constexpr int kTmemCols = 512;
+constexpr int kMiscBytes = 8192;                 // barriers + reduction scratch at the head of smem
+constexpr int kMaxStages = 12;
+constexpr int kHStages = 4;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct FusedParams {
+  int num_kb;       // d / 64
+  int num_tiles;    // ceil(V / 128)
+  int stages;       // W ring depth
+  int tmem_tiles;   // tiles resident in TMEM
+  int R;            // B * (M + 1)
+  uint32_t off_h;   // byte offsets inside dynamic smem (from the 1024-aligned base)
+  uint32_t off_ovf;
+  uint32_t off_w;
+};
+
+// ------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (unsigned it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (it > 128) {
+      __nanosleep(64);
+      if (*abort_flag) return false;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// K-major, 128-byte swizzle shared-memory matrix descriptor: start address, stride between
+// 8-row groups = 1024 bytes, descriptor version 1, layout type 2 (SWIZZLE_128B).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(1024u >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor, kind::f16: D = f32, A = B = bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t make_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float tmem_ld1(uint32_t taddr) {
+  uint32_t r;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  return __uint_as_float(r);
+}
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Grid barrier on a global counter; thread 0 of the epilogue group calls it. Cooperative launch
+// guarantees co-residency; the spin is bounded all the same.
+__device__ __forceinline__ bool grid_arrive_and_wait(unsigned* counter, unsigned expected, volatile int* abort_flag) {
+  __threadfence();
+  atomicAdd(counter, 1u);
+  for (unsigned it = 0; it < kSpinLimit; ++it) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+    if (v >= expected) return true;
+    __nanosleep(40);
+    if (*abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// ------------------------------------------------------------------------------ shared scratch
+template <int N_PAD>
+struct Misc {
+  uint64_t full_w[kMaxStages], empty_w[kMaxStages];
+  uint64_t full_h[kHStages], empty_h[kHStages];
+  uint64_t acc_full[2];
+  uint64_t drained;
+  uint32_t tmem_base;
+  int abort_flag;
+  float wmax[4][N_PAD];
+  float wsum[4][N_PAD];
+  float cta_max[N_PAD];
+  float lse[N_PAD];       // log-normaliser of every row (all CTAs compute the same values)
+  float rmax[N_PAD];
+  float qlse[N_PAD];
+  int x_row[N_PAD];       // drafted token of row r (rows j < M), -1 otherwise
+  int sel_row[N_PAD];
+  int sel_kind[N_PAD];
+  float sel_lse_p[N_PAD];
+  float sel_lse_q[N_PAD];
+  float sel_u[N_PAD];
+  double wd[2][4];
+  int cand[4];
+  int lastpos[4];
+};
+
+// logit of (tile i, this thread's lane, row r): from TMEM or from the overflow copy in smem
+template <int N_PAD>
+__device__ __forceinline__ void load_chunk(int i, int c0, int n_ovf, uint32_t tmem_lane_base, const float* ovf, int tid,
+                                           float* v) {
+  if (i < n_ovf) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) v[k] = ovf[((size_t)i * N_PAD + c0 + k) * kVocabTile + tid];
+  } else {
+    tmem_ld16(tmem_lane_base + (uint32_t)((i - n_ovf) * N_PAD + c0), v);
+  }
+}
+template <int N_PAD>
+__device__ __forceinline__ float load_one(int i, int r, int n_ovf, uint32_t tmem_lane_base, const float* ovf, int tid) {
+  if (i < n_ovf) return ovf[((size_t)i * N_PAD + r) * kVocabTile + tid];
+  return tmem_ld1(tmem_lane_base + (uint32_t)((i - n_ovf) * N_PAD + r));
+}
+
+template <int N_PAD>
+__global__ void __launch_bounds__(kThreads, 1)
+fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, CallParams cp,
+                    Workspace ws, const __nv_bfloat16* __restrict__ H, const __nv_bfloat16* __restrict__ wj,
+                    FusedParams fp) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  Misc<N_PAD>& ms = *reinterpret_cast<Misc<N_PAD>*>(smem);
+  static_assert(sizeof(Misc<N_PAD>) <= kMiscBytes, "misc block too large");
+  const uint32_t sH = smem_u32(smem + fp.off_h);
+  const uint32_t sW = smem_u32(smem + fp.off_w);
+  const float* ovf = reinterpret_cast<const float*>(smem + fp.off_ovf);
+  float* ovf_w = reinterpret_cast<float*>(smem + fp.off_ovf);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = blockIdx.x, G = gridDim.x;
+  volatile int* abort_flag = &ms.abort_flag;
+
+  // vocabulary tiles of this CTA
+  const int base = fp.num_tiles / G, rem = fp.num_tiles % G;
+  const int T = base + (cta < rem ? 1 : 0);
+  const int t0 = cta * base + min(cta, rem);
+  const int n_ovf = max(0, T - fp.tmem_tiles);   // first n_ovf tiles go through TMEM into smem
+  const int R = fp.R, M = cp.M, V = cp.V;
+  const int BM = cp.B * M;
+
+  if (tid == 0) {
+    for (int s = 0; s < fp.stages; ++s) { mbar_init(smem_u32(&ms.full_w[s]), 1); mbar_init(smem_u32(&ms.empty_w[s]), 1); }
+    for (int s = 0; s < kHStages; ++s) { mbar_init(smem_u32(&ms.full_h[s]), 1); mbar_init(smem_u32(&ms.empty_h[s]), 1); }
+    mbar_init(smem_u32(&ms.acc_full[0]), 1);
+    mbar_init(smem_u32(&ms.acc_full[1]), 1);
+    mbar_init(smem_u32(&ms.drained), 1);
+    ms.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid < N_PAD) {
+    int x = -1;
+    if (tid < R) {
+      const int b = tid / (M + 1), j = tid % (M + 1);
+      if (j < M) {
+        x = cp.draft_tokens[b * M + j];
+        if (x < 0 || x >= V) { set_status(ws.status, JD_ERR_BAD_TOKEN); x = min(max(x, 0), V - 1); }
+      }
+    }
+    ms.x_row[tid] = x;
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ms.tmem_base)),
+                 "r"((uint32_t)kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ms.tmem_base;
+
+  // group 0 = the n_ovf overflow tiles (if any), group 1 = the TMEM-resident tiles
+  const int g_begin[2] = {0, n_ovf};
+  const int g_end[2] = {n_ovf, T};
+
+  if (warp == 4 && lane == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    const uint64_t pol_w = policy_evict_first(), pol_h = policy_evict_last();
+    int ws_i = 0, hs_i = 0;
+    uint32_t wph = 0, hph = 0;
+    bool ok = true;
+    for (int g = 0; g < 2 && ok; ++g) {
+      if (g_begin[g] == g_end[g]) continue;
+      for (int kb = 0; kb < fp.num_kb && ok; ++kb) {
+        ok = mbar_wait(smem_u32(&ms.empty_h[hs_i]), hph ^ 1u, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(smem_u32(&ms.full_h[hs_i]), N_PAD * 128);
+        tma_load_2d(sH + hs_i * (N_PAD * 128), &tmH, smem_u32(&ms.full_h[hs_i]), kb * kBlockK, 0, pol_h);
+        if (++hs_i == kHStages) { hs_i = 0; hph ^= 1u; }
+        for (int i = g_begin[g]; i < g_end[g]; ++i) {
+          ok = mbar_wait(smem_u32(&ms.empty_w[ws_i]), wph ^ 1u, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(smem_u32(&ms.full_w[ws_i]), kWStageBytes);
+          tma_load_2d(sW + ws_i * kWStageBytes, &tmW, smem_u32(&ms.full_w[ws_i]), kb * kBlockK, (t0 + i) * kVocabTile,
+                      pol_w);
+          if (++ws_i == fp.stages) { ws_i = 0; wph ^= 1u; }
+        }
+      }
+    }
+    if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
+  } else if (warp == 5 && lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer
+    const uint32_t idesc = make_idesc(N_PAD);
+    int ws_i = 0, hs_i = 0;
+    uint32_t wph = 0, hph = 0;
+    bool ok = true;
+    for (int g = 0; g < 2 && ok; ++g) {
+      if (g_begin[g] == g_end[g]) continue;
+      if (g == 1 && n_ovf > 0) {   // the overflow tiles must have left TMEM before it is reused
+        ok = mbar_wait(smem_u32(&ms.drained), 0u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      for (int kb = 0; kb < fp.num_kb && ok; ++kb) {
+        ok = mbar_wait(smem_u32(&ms.full_h[hs_i]), hph, abort_flag);
+        if (!ok) break;
+        const uint32_t hb = sH + hs_i * (N_PAD * 128);
+        for (int i = g_begin[g]; i < g_end[g]; ++i) {
+          ok = mbar_wait(smem_u32(&ms.full_w[ws_i]), wph, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t wb = sW + ws_i * kWStageBytes;
+          const uint32_t dcol = tmem_base + (uint32_t)((i - g_begin[g]) * N_PAD);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 16; ++k) {
+            umma_bf16(dcol, make_smem_desc(wb + k * 32), make_smem_desc(hb + k * 32), idesc,
+                      (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&ms.empty_w[ws_i]));
+          if (++ws_i == fp.stages) { ws_i = 0; wph ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&ms.empty_h[hs_i]));
+        if (++hs_i == kHStages) { hs_i = 0; hph ^= 1u; }
+      }
+      if (ok) umma_commit(smem_u32(&ms.acc_full[g]));
+    }
+    if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
+  } else if (warp < 4) {
+    // ------------------------------------------------------------------ epilogue warps
+    const uint32_t tmem_lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    bool ok = true;
+
+    // (a) overflow tiles: TMEM -> smem as soon as their accumulation is complete
+    if (n_ovf > 0) {
+      ok = mbar_wait(smem_u32(&ms.acc_full[0]), 0u, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        for (int i = 0; i < n_ovf; ++i) {
+#pragma unroll
+          for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+            float v[16];
+            tmem_ld16(tmem_lane_base + (uint32_t)(i * N_PAD + c0), v);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) ovf_w[((size_t)i * N_PAD + c0 + k) * kVocabTile + tid] = v[k];
+          }
+        }
+        tc_fence_before();
+      }
+      epi_sync();
+      if (tid == 0) mbar_arrive(smem_u32(&ms.drained));
+    }
+
+    // (b) while W streams: draft-row statistics over this CTA's vocabulary slice, judge dots
+    const int v_lo = t0 * kVocabTile, v_hi = min(V, (t0 + T) * kVocabTile);
+    for (int bm = warp; bm < BM; bm += 4) {
+      const float* row = cp.draft_logits + (size_t)bm * V;
+      float m = -INFINITY, s = 0.f;
+      for (int v = v_lo + lane; v < v_hi; v += 32) {
+        const float xv = __ldg(row + v);
+        if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
+        else if (xv != -INFINITY) s += __expf(xv - m);
+      }
+      ms_warp_reduce(m, s);
+      if (lane == 0) {
+        ws.qpart_max[(size_t)bm * G + cta] = m;
+        ws.qpart_sum[(size_t)bm * G + cta] = s;
+        const int b = bm / M, j = bm % M;
+        const int x = ms.x_row[b * (M + 1) + j];
+        if (x >= v_lo && x < v_hi) ws.qgath[bm] = row[x];
+      }
+    }
+    for (int bm = cta * 4 + warp; bm < BM; bm += G * 4) {
+      const int b = bm / M, j = bm % M;
+      const uint4* h4 = reinterpret_cast<const uint4*>(H + ((size_t)b * (M + 1) + j + 1) * cp.d);
+      const uint4* w4 = reinterpret_cast<const uint4*>(wj);
+      float acc = 0.f;
+      for (int k = lane; k < cp.d / 8; k += 32) {
+        const uint4 hv = __ldg(h4 + k), wv = __ldg(w4 + k);
+        const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+        const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 a = __bfloat1622float2(hp[e]), c = __bfloat1622float2(wp[e]);
+          acc = fmaf(a.x, c.x, acc);
+          acc = fmaf(a.y, c.y, acc);
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (lane == 0) ws.judge_logit[bm] = acc;
+    }
+
+    // (c) wait for the logits of the resident tiles
+    if (ok && T > n_ovf) ok = mbar_wait(smem_u32(&ms.acc_full[1]), 0u, abort_flag);
+    tc_fence_after();
+    epi_sync();
+    ok = ok && (*abort_flag == 0);
+
+    // (d) per-row max over this CTA's slice, and the gather of the drafted tokens' logits
+    {
+      float m[N_PAD];
+#pragma unroll
+      for (int r = 0; r < N_PAD; ++r) m[r] = -INFINITY;
+      if (ok) {
+        for (int i = 0; i < T; ++i) {
+          const int vg = (t0 + i) * kVocabTile + tid;
+          const bool valid = vg < V;
+#pragma unroll
+          for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+            float v[16];
+            load_chunk<N_PAD>(i, c0, n_ovf, tmem_lane_base, ovf, tid, v);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+              if (valid) {
+                m[c0 + k] = fmaxf(m[c0 + k], v[k]);
+                if (ms.x_row[c0 + k] == vg) ws.gath[c0 + k] = v[k];
+              }
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < N_PAD; ++r) {
+        float x = m[r];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+        if (lane == 0) ms.wmax[warp][r] = x;
+      }
+    }
+    epi_sync();
+    if (tid < N_PAD) ms.cta_max[tid] = fmaxf(fmaxf(ms.wmax[0][tid], ms.wmax[1][tid]), fmaxf(ms.wmax[2][tid], ms.wmax[3][tid]));
+    epi_sync();
+
+    // (e) per-row sum exp(L - cta max)
+    {
+      float s[N_PAD];
+#pragma unroll
+      for (int r = 0; r < N_PAD; ++r) s[r] = 0.f;
+      if (ok) {
+        for (int i = 0; i < T; ++i) {
+          const bool valid = (t0 + i) * kVocabTile + tid < V;
+#pragma unroll
+          for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+            float v[16];
+            load_chunk<N_PAD>(i, c0, n_ovf, tmem_lane_base, ovf, tid, v);
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+              if (valid) s[c0 + k] += exp2f((v[k] - ms.cta_max[c0 + k]) * kLog2e);
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < N_PAD; ++r) {
+        float x = s[r];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        if (lane == 0) ms.wsum[warp][r] = x;
+      }
+    }
+    epi_sync();
+    if (tid < R) {
+      ws.part_max[(size_t)tid * G + cta] = ms.cta_max[tid];
+      ws.part_sum[(size_t)tid * G + cta] = (ms.wsum[0][tid] + ms.wsum[1][tid]) + (ms.wsum[2][tid] + ms.wsum[3][tid]);
+    }
+    __threadfence();
+    epi_sync();
+
+    // ------------------------------------------------------------------ grid barrier 1
+    if (tid == 0) {
+      if (!ok || !grid_arrive_and_wait(ws.barrier + 0, (unsigned)G, abort_flag)) {
+        *abort_flag = 1;
+        set_status(ws.status, JD_ERR_TIMEOUT);
+      }
+    }
+    epi_sync();
+    ok = (*abort_flag == 0);
+
+    if (ok) {
+      // (f) fold the per-CTA statistics of every row (every CTA computes the same numbers)
+      for (int r = warp; r < R; r += 4) {
+        float m = -INFINITY, s = 0.f;
+        for (int c = lane; c < G; c += 32)
+          ms_combine(m, s, __ldcg(ws.part_max + (size_t)r * G + c), __ldcg(ws.part_sum + (size_t)r * G + c));
+        ms_warp_reduce(m, s);
+        if (lane == 0) {
+          const float lse = m + logf(s);
+          ms.rmax[r] = m;
+          ms.lse[r] = lse;
+          if (cta == 0) {
+            if (cp.row_max_out) cp.row_max_out[r] = m;
+            if (cp.row_lse_out) cp.row_lse_out[r] = lse;
+          }
+        }
+      }
+      for (int bm = warp; bm < BM; bm += 4) {
+        float m = -INFINITY, s = 0.f;
+        for (int c = lane; c < G; c += 32)
+          ms_combine(m, s, __ldcg(ws.qpart_max + (size_t)bm * G + c), __ldcg(ws.qpart_sum + (size_t)bm * G + c));
+        ms_warp_reduce(m, s);
+        if (lane == 0) ms.qlse[bm] = m + logf(s);
+      }
+    }
+    epi_sync();
+    if (ok) {
+      // (g) tests, mask, accepted prefix (Eq. 4; Sec. 4.1): one warp per sequence
+      Workspace lw = ws;
+      lw.row_lse = ms.lse;
+      lw.q_lse = ms.qlse;
+      lw.sel_row = ms.sel_row;
+      lw.sel_kind = ms.sel_kind;
+      lw.sel_lse_p = ms.sel_lse_p;
+      lw.sel_lse_q = ms.sel_lse_q;
+      lw.sel_u = ms.sel_u;
+      for (int b = warp; b < cp.B; b += 4) decide_sequence(cp, lw, b, cta == 0);
+    }
+    epi_sync();
+
+    // (h) mass of the sampling weights of each selected row over this CTA's slice
+    if (ok) {
+      for (int b = 0; b < cp.B; ++b) {
+        const int row = ms.sel_row[b], kind = ms.sel_kind[b];
+        const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
+        const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;   // used only when kind == 0
+        double sr = 0.0, sp = 0.0;
+        for (int i = 0; i < T; ++i) {
+          const int vg = (t0 + i) * kVocabTile + tid;
+          const float logit = load_one<N_PAD>(i, row, n_ovf, tmem_lane_base, ovf, tid);
+          if (vg < V) {
+            float p, r;
+            sample_weights(logit, lse_p, kind, kind == 0 ? __ldg(dlrow + vg) : 0.f, lse_q, p, r);
+            sr += (double)r;
+            sp += (double)p;
+          }
+        }
+        sr = warp_sum_double(sr);
+        sp = warp_sum_double(sp);
+        if (lane == 0) { ms.wd[0][warp] = sr; ms.wd[1][warp] = sp; }
+        epi_sync();
+        if (tid == 0) {
+          ws.mass_r[(size_t)b * G + cta] = (ms.wd[0][0] + ms.wd[0][1]) + (ms.wd[0][2] + ms.wd[0][3]);
+          ws.mass_p[(size_t)b * G + cta] = (ms.wd[1][0] + ms.wd[1][1]) + (ms.wd[1][2] + ms.wd[1][3]);
+        }
+        epi_sync();
+      }
+    }
+    __threadfence();
+    epi_sync();
+
+    // ------------------------------------------------------------------ grid barrier 2
+    if (tid == 0) {
+      if (!ok || !grid_arrive_and_wait(ws.barrier + 1, (unsigned)G, abort_flag)) {
+        *abort_flag = 1;
+        set_status(ws.status, JD_ERR_TIMEOUT);
+      }
+    }
+    epi_sync();
+    ok = (*abort_flag == 0);
+
+    // (i) inverse CDF in ascending token id: find the owning CTA, then the token inside it
+    if (ok) {
+      for (int b = 0; b < cp.B; ++b) {
+        // every warp scans the per-CTA masses in the same order: lane l owns CTAs [l*per, (l+1)*per)
+        const int per = (G + 31) / 32;
+        const double* mass = ws.mass_r + (size_t)b * G;
+        bool use_p = false;
+        double chunk = 0.0;
+        for (int c = lane * per; c < min(G, (lane + 1) * per); ++c) chunk += __ldcg(mass + c);
+        double total = warp_sum_double(chunk);
+        if (!(total > 0.0)) {   // identically zero residual: draw from p
+          use_p = true;
+          mass = ws.mass_p + (size_t)b * G;
+          chunk = 0.0;
+          for (int c = lane * per; c < min(G, (lane + 1) * per); ++c) chunk += __ldcg(mass + c);
+        }
+        // exclusive prefix of the lane chunks (sequential over lanes, identical in every warp)
+        double excl = 0.0, run = 0.0;
+        for (int l = 0; l < 32; ++l) {
+          const double cl = __shfl_sync(0xffffffffu, chunk, l);
+          if (l == lane) excl = run;
+          run += cl;
+        }
+        total = run;
+        const double Tt = (double)ms.sel_u[b] * total;
+        // owner = first CTA whose inclusive prefix exceeds T, else the last CTA with mass
+        int owner = -1, last_mass = -1;
+        double my_prefix = 0.0;   // exclusive prefix of the owner, valid in the lane that finds it
+        {
+          double c = excl;
+          for (int cc = lane * per; cc < min(G, (lane + 1) * per); ++cc) {
+            const double mc = __ldcg(mass + cc);
+            if (mc > 0.0) last_mass = cc;
+            if (owner < 0 && c + mc > Tt) { owner = cc; my_prefix = c; }
+            c += mc;
+          }
+        }
+        const unsigned found = __ballot_sync(0xffffffffu, owner >= 0);
+        double owner_prefix;
+        if (found) {
+          const int src = __ffs(found) - 1;
+          owner = __shfl_sync(0xffffffffu, owner, src);
+          owner_prefix = __shfl_sync(0xffffffffu, my_prefix, src);
+        } else {
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) last_mass = max(last_mass, __shfl_xor_sync(0xffffffffu, last_mass, o));
+          owner = last_mass;
+          owner_prefix = -1.0;   // marks the "T beyond the total" fallback
+        }
+        if (owner != cta) continue;   // uniform over the CTA: every warp computed the same owner
+
+        const int row = ms.sel_row[b];
+        const int kind = use_p ? 1 : ms.sel_kind[b];
+        const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
+        const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;
+        const bool beyond = owner_prefix < 0.0;
+        double c_tile = beyond ? 0.0 : owner_prefix;
+        int token = -1, last_token = -1;
+        for (int i = 0; i < T && token < 0; ++i) {
+          const int vg = (t0 + i) * kVocabTile + tid;
+          const float logit = load_one<N_PAD>(i, row, n_ovf, tmem_lane_base, ovf, tid);
+          float p = 0.f, r = 0.f;
+          if (vg < V) sample_weights(logit, lse_p, kind, kind == 0 ? __ldg(dlrow + vg) : 0.f, lse_q, p, r);
+          // ordered inclusive scan over the 128 lanes of the tile, in double
+          double incl = (double)r;
+#pragma unroll
+          for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+          }
+          if (lane == 31) ms.wd[0][warp] = incl;
+          const unsigned pos = __ballot_sync(0xffffffffu, r > 0.f);
+          if (lane == 0) ms.lastpos[warp] = pos ? (31 - __clz(pos)) : -1;
+          epi_sync();
+          double off = c_tile;
+          for (int w = 0; w < warp; ++w) off += ms.wd[0][w];
+          const double tile_total = (ms.wd[0][0] + ms.wd[0][1]) + (ms.wd[0][2] + ms.wd[0][3]);
+          const unsigned hit = beyond ? 0u : __ballot_sync(0xffffffffu, off + incl > Tt);
+          if (lane == 0) ms.cand[warp] = hit ? (__ffs(hit) - 1) : -1;
+          epi_sync();
+          for (int w = 0; w < 4; ++w) {
+            if (token < 0 && ms.cand[w] >= 0) token = (t0 + i) * kVocabTile + w * 32 + ms.cand[w];
+            if (ms.lastpos[w] >= 0) last_token = (t0 + i) * kVocabTile + w * 32 + ms.lastpos[w];
+          }
+          c_tile += tile_total;
+          epi_sync();
+        }
+        if (token < 0) token = last_token;   // rounding at the upper edge: the last token with mass
+        if (tid == 0) cp.next_token[b] = token < 0 ? 0 : token;
+      }
+    }
+    tc_fence_before();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncthreads();
+  if (ms.abort_flag) {
+    // give copies that may still be in flight time to land before the shared memory is released
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);
+    __syncthreads();
+  }
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols)
+                 : "memory");
+  }
+}
+
+template <int N_PAD>
+cudaError_t launch_fused(const CUtensorMap& tmW, const CUtensorMap& tmH, const CallParams& cp, const Workspace& ws,
+                         const void* H, const void* wj, const FusedParams& fp, const FusedPlan& plan,
+                         cudaStream_t st) {
+  auto kern = fused_verify_kernel<N_PAD>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
+  if (e != cudaSuccess) return e;
+  const __nv_bfloat16* Hp = (const __nv_bfloat16*)H;
+  const __nv_bfloat16* wp = (const __nv_bfloat16*)wj;
+  void* args[] = {(void*)&tmW, (void*)&tmH, (void*)&cp, (void*)&ws, (void*)&Hp, (void*)&wp, (void*)&fp};
+  return cudaLaunchCooperativeKernel((const void*)kern, dim3(plan.num_ctas), dim3(kThreads), args, plan.smem_bytes,
+                                     st);
+}
+
+}  // namespace
+
+bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan) {
+  if (dtype != JD_DTYPE_BF16 || d % kBlockK != 0 || d < kBlockK || R < 1 || R > 96) return false;
+  if (num_sms < 1 || num_sms > kMaxCtas) return false;
+  const int n_pad = (R + 15) / 16 * 16;
+  const int num_tiles = (V + kVocabTile - 1) / kVocabTile;
+  const int max_tiles = (num_tiles + num_sms - 1) / num_sms;
+  const int tmem_tiles = std::min(max_tiles, kTmemCols / n_pad);
+  const int n_ovf = max_tiles - tmem_tiles;
+  if (n_ovf > tmem_tiles) return false;   // the overflow group itself must fit in TMEM
+  const size_t fixed = 1024 /*alignment slack*/ + kMiscBytes + (size_t)kHStages * n_pad * 128 +
+                       (size_t)n_ovf * kVocabTile * n_pad * 4;
+  const size_t budget = 227 * 1024;
+  if (fixed + 4 * (size_t)kWStageBytes > budget) return false;
+  int stages = (int)((budget - fixed) / kWStageBytes);
+  stages = std::min(stages, kMaxStages);
+  if (plan) {
+    plan->num_ctas = num_sms;
+    plan->n_pad = n_pad;
+    plan->max_tiles = max_tiles;
+    plan->tmem_tiles = tmem_tiles;
+    plan->stages = stages;
+    plan->smem_bytes = fixed + (size_t)stages * kWStageBytes;
+  }
+  return true;
+}
+
+int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
+              const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err) {
+  FusedParams fp;
+  fp.num_kb = cp.d / kBlockK;
+  fp.num_tiles = (cp.V + kVocabTile - 1) / kVocabTile;
+  fp.stages = plan.stages;
+  fp.tmem_tiles = plan.tmem_tiles;
+  fp.R = cp.B * (cp.M + 1);
+  fp.off_h = kMiscBytes;
+  fp.off_ovf = fp.off_h + kHStages * plan.n_pad * 128;
+  const int n_ovf = plan.max_tiles - plan.tmem_tiles;
+  fp.off_w = fp.off_ovf + (uint32_t)n_ovf * kVocabTile * plan.n_pad * 4;
+  fp.off_w = (fp.off_w + 1023u) & ~1023u;
+  cudaError_t e;
+  switch (plan.n_pad) {
+    case 16: e = launch_fused<16>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
+    case 32: e = launch_fused<32>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
+    case 48: e = launch_fused<48>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
+    case 64: e = launch_fused<64>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
+    case 80: e = launch_fused<80>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
+    case 96: e = launch_fused<96>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
+    default: e = cudaErrorInvalidValue; break;
+  }
+  *err = e;
+  return e == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace jd

@@ -190,3 +190,52 @@ def test_host_buffer_entry_point_matches_device_call_and_is_repeatable():
         assert np.array_equal(d1[k], d2[k]), k              # run-to-run determinism
         assert np.array_equal(d1[k], h1[k]), k
     ver.close()
+
+
+# ------------------------------------------------------------------ fused tensor-core variant
+FUSED_SHAPES = [
+    (1, 1, 64, 130),          # two vocabulary tiles, ragged tail, n_pad 16
+    (2, 3, 64, 1000),         # only 8 of the CTAs own a tile
+    (1, 8, 256, 128256),      # 8B-head rows: n_pad 16, seven tiles per CTA
+    (1, 25, 192, 50000),      # n_pad 32, ragged last tile
+    (3, 20, 128, 40000),      # n_pad 64
+    (4, 16, 128, 128256),     # 70B-head rows: n_pad 80, one tile per CTA overflows to shared memory
+    (5, 15, 128, 128256 + 77),  # same with a ragged last tile
+    (6, 15, 64, 128256),      # n_pad 96, two overflow tiles
+]
+
+
+@pytest.mark.parametrize("B,M,d,V", FUSED_SHAPES)
+def test_fused_variant_parity(B, M, d, V):
+    wl = I.CONFIGS[2].scaled("fused-%d-%d-%d-%d" % (B, M, d, V), B=B, M=M, d=d, V=V)
+    rep = run_case(wl, 3, variant="fused", seeds=[0, 1], expect_variant="fused")
+    assert rep.sequences == 6 * B
+
+
+def test_fused_matches_simt_variant_on_device():
+    wl = I.CONFIGS[2].scaled("x", B=4, M=16, d=256, V=128256)
+    inp = I.make_inputs(wl, 2)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    for seed in range(3):
+        a = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, seed, "judge_or_standard", variant="fused"))
+        b = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, seed, "judge_or_standard", variant="simt"))
+        a2 = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, seed, "judge_or_standard", variant="fused"))
+        for k in a:
+            assert np.array_equal(a[k], a2[k]), k                     # repeatable bit for bit
+        assert np.array_equal(a["accept_len"], b["accept_len"])
+        assert np.array_equal(a["masks"], b["masks"])
+        assert np.allclose(a["row_lse"], b["row_lse"], rtol=0, atol=1e-4)
+        assert np.allclose(a["p_draft"], b["p_draft"], rtol=1e-4)
+    ver.close()
+
+
+def test_fused_unsupported_shapes_are_refused_not_faked():
+    from paper_2501_19309_b200 import jd
+    wl = I.CONFIGS[2].scaled("x", B=8, M=16, d=128, V=2000)           # 136 rows > 96
+    inp = I.make_inputs(wl, 2)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    a, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, variant="fused")
+    assert jd.jd_verify(ver.h, a) == jd.JD_ERR_UNSUPPORTED
+    ver.close()

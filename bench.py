@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the fused verification step (jd_verify) on synthetic Llama-3.1-shaped heads.
+
+One step = one verification call (LM head -> softmax -> tests -> prefix -> next token) over one
+synthetic draft block.  Prints ONE JSON line:
+
+  value     verified tokens/s (B*M per call), inputs resident in device memory, CUDA-event time
+  e2e       the same through jd_verify_host: pinned host inputs copied in, outputs copied back
+  roofline  achieved (W bytes + H bytes) / kernel time against the measured HBM copy bandwidth
+            (or 2*R*V*d flop / time against the measured bf16 peak when that bound is larger)
+  cpu_baseline  the float64 CPU checker timed on a bounded sample of the same workload
+
+`--impl reference` times the CPU checker alone (rank 0 only).
+With --gpus N > 1 (launched under torchrun) every rank runs an independent replica: the path has
+no exchange step, so the aggregate is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2501_19309_b200 import inputs as I  # noqa: E402
+
+METRIC = "verified_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes (read + write) per launch of the fused kernel from an ncu capture, per workload;
+# None until captured for the kernel as it stands.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.rows = []
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [t.strip() for t in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, which: str) -> dict:
+    bytes_alg = wl.V * wl.d * 2 + wl.R * wl.d * 2            # W once + H once
+    flops = 2.0 * wl.R * wl.V * wl.d
+    tf_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    t_bytes = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+    t_flops = flops / (tf_peak * 1e12)
+    traffic = NCU_TRAFFIC_BYTES.get(wl.name)
+    if t_bytes >= t_flops:
+        ach = bytes_alg / (kernel_ms * 1e-3) / 1e9
+        return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "peak_source": which,
+                "algorithmic_bytes": bytes_alg, "kernel_ms": kernel_ms}
+    ach = flops / (kernel_ms * 1e-3) / 1e12
+    return {"bound": "tensor", "achieved": ach, "peak": tf_peak, "unit": "TFLOP/s", "frac": ach / tf_peak,
+            "traffic": traffic, "peak_source": which, "algorithmic_flops": flops, "kernel_ms": kernel_ms}
+
+
+def oracle_step(inp: I.Inputs, seed: int, sequences):
+    from oracle import jd_oracle as O
+    return O.jd_oracle_verify(inp.W, inp.w_judge, inp.b_judge, inp.H, inp.draft_tokens, inp.draft_logits,
+                              inp.tau, seed, "judge_or_standard", sequences=sequences)
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 1) for d in threadpool_info() if d.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def time_oracle(inp: I.Inputs, steps: int, budget_s: float = 25.0) -> dict:
+    """The checker as it stands on a bounded sample: whole sequences b = 0, 1, ... of the workload."""
+    wl = inp.wl
+    t0 = time.perf_counter()
+    oracle_step(inp, 0, [0])
+    one = time.perf_counter() - t0
+    nseq = int(max(1, min(wl.B, budget_s / max(one, 1e-3) / max(steps, 1))))
+    seqs = list(range(nseq))
+    t0 = time.perf_counter()
+    for s in range(steps):
+        oracle_step(inp, s, seqs)
+    dt = time.perf_counter() - t0
+    return {"value": nseq * wl.M * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+            "sample": "%d step(s) x %d of %d sequences (%d rows x V=%d x d=%d each), float64 numpy" %
+                      (steps, nseq, wl.B, wl.M + 1, wl.V, wl.d),
+            "seconds": dt}
+
+
+def run_reference(args, wl) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = I.make_inputs(wl, 0)
+    steps = max(1, min(args.steps, 3))
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(inp, 0, [0])
+    r = time_oracle(inp, steps, budget_s=60.0)
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": r["seconds"] / steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": wl.name, "B": wl.B, "M": wl.M, "d": wl.d, "V": wl.V},
+            "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
+    """Times K device-resident calls and K_e2e host-buffer calls of one workload on this rank."""
+    inp = I.make_inputs(wl, data_seed)
+    W = torch.from_numpy(inp.W).view(torch.bfloat16).to(device)
+    H = torch.from_numpy(inp.H).view(torch.bfloat16).to(device)
+    w = torch.from_numpy(inp.w_judge).view(torch.bfloat16).to(device)
+    x = torch.from_numpy(inp.draft_tokens).to(device)
+    dl = torch.from_numpy(inp.draft_logits).to(device)
+    ver = jd.Verifier(wl.B, wl.M, wl.d, wl.V, "bf16", device.index)
+    ver.set_head(W, w, inp.b_judge)
+    out = ver.alloc_outputs(wl.B, wl.M)
+    a_args = [ver.make_args(H, x, dl, inp.tau, s, "judge_or_standard", out=out)[0] for s in range(8)]
+    stream = torch.cuda.current_stream(device)
+
+    def step(i):
+        st = jd.jd_verify(ver.h, a_args[i % 8], stream.cuda_stream)
+        if st != jd.JD_OK:
+            raise jd.JdError(st, "jd_verify")
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize(device)
+    assert ver.device_status() == jd.JD_OK
+    variant, launches = ver.launch_info()
+
+    sampler = ClockSampler(device.index) if sample_clocks else None
+    if sampler:
+        time.sleep(0.6)          # let the sampler start
+    if args.dist:
+        torch.distributed.barrier()
+    torch.cuda.synchronize(device)
+    K = args.steps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(K):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize(device)
+    if args.dist:
+        torch.distributed.barrier()
+    total_ms = e0.elapsed_time(e1)
+    # per-call distribution on a short second pass (events between calls)
+    Kp = min(K, 200)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(Kp + 1)]
+    evs[0].record(stream)
+    for i in range(Kp):
+        step(i)
+        evs[i + 1].record(stream)
+    torch.cuda.synchronize(device)
+    per = [evs[i].elapsed_time(evs[i + 1]) for i in range(Kp)]
+    clocks = sampler.stop() if sampler else None
+    assert ver.device_status() == jd.JD_OK
+    accepted = out["accept_len"].cpu().numpy()
+
+    # end to end: pinned host buffers in, outputs back, every step
+    hH = torch.from_numpy(inp.H).view(torch.bfloat16).pin_memory()
+    hx = torch.from_numpy(inp.draft_tokens).pin_memory()
+    hdl = torch.from_numpy(inp.draft_logits).pin_memory()
+    hout = ver.alloc_outputs(wl.B, wl.M, host=True)
+    h_args = [ver.make_args(hH, hx, hdl, inp.tau, s, "judge_or_standard", out=hout, host=True)[0] for s in range(8)]
+    Ke = max(3, min(K, args.e2e_steps))
+    for i in range(3):
+        jd.jd_verify_host(ver.h, h_args[i % 8], stream.cuda_stream)
+    torch.cuda.synchronize(device)
+    if args.dist:
+        torch.distributed.barrier()
+    t0 = time.perf_counter()
+    for i in range(Ke):
+        st = jd.jd_verify_host(ver.h, h_args[i % 8], stream.cuda_stream)
+        if st != jd.JD_OK:
+            raise jd.JdError(st, "jd_verify_host")
+    torch.cuda.synchronize(device)
+    e2e_s = time.perf_counter() - t0
+    h2d = hH.numel() * 2 + hx.numel() * 4 + hdl.numel() * 4
+    d2h = sum(hout[k].numel() * hout[k].element_size() for k in hout)
+    ver.close()
+    res = dict(total_ms=total_ms, median_ms=statistics.median(per), min_ms=min(per), mean_ms=total_ms / K,
+               variant=variant, launches=launches, clocks=clocks, e2e_s=e2e_s, e2e_steps=Ke, h2d=h2d, d2h=d2h,
+               mean_accept=float(accepted.mean()), inp=inp)
+    del W, H, dl
+    torch.cuda.empty_cache()
+    return res
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, help="workload id of the headline line (1..4)")
+    ap.add_argument("--others", default="2,3", help="comma list of further workloads summarised in the same line")
+    ap.add_argument("--e2e-steps", type=int, default=200)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    wl = I.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    from paper_2501_19309_b200 import jd
+    jd.load()   # raises if the CUDA library is missing: there is no other path
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    args.dist = world > 1
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    if args.dist:
+        torch.distributed.init_process_group("nccl", device_id=device)
+
+    peaks, which = load_peaks()
+    res = measure_workload(wl, args, torch, jd, device, data_seed=rank, sample_clocks=True)
+
+    # max over ranks of the timed region, sum of the units
+    t = torch.tensor([res["total_ms"], res["e2e_s"]], dtype=torch.float64, device=device)
+    if args.dist:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    total_ms, e2e_s = float(t[0]), float(t[1])
+    K = args.steps
+    tokens_per_step = wl.B * wl.M
+    value = world * tokens_per_step * K / (total_ms * 1e-3)
+    e2e_value = world * tokens_per_step * res["e2e_steps"] / e2e_s
+
+    others = {}
+    if rank == 0 and args.others:
+        small = argparse.Namespace(**vars(args))
+        small.dist = False
+        for cid in [int(c) for c in args.others.split(",") if c.strip()]:
+            if cid == args.config or cid not in I.CONFIGS:
+                continue
+            owl = I.CONFIGS[cid]
+            small.steps = max(50, min(args.steps, 300))
+            r = measure_workload(owl, small, torch, jd, device, data_seed=0, sample_clocks=False)
+            others[owl.name] = {
+                "B": owl.B, "M": owl.M, "d": owl.d, "V": owl.V, "ms_per_step": r["mean_ms"],
+                "median_ms": r["median_ms"], "value": owl.B * owl.M / (r["mean_ms"] * 1e-3), "unit": UNIT,
+                "variant": r["variant"], "steps": small.steps,
+                "roofline": roofline_of(owl, peaks, r["mean_ms"], sustained=r["mean_ms"] * small.steps > 1000, which=which)}
+
+    if rank == 0:
+        cpu = None
+        if not args.no_cpu_baseline:
+            c = time_oracle(res["inp"], 1)
+            cpu = {k: c[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "M": wl.M, "d": wl.d, "V": wl.V, "mode": "judge_or_standard",
+                       "variant": {1: "simt", 2: "fused", 3: "batched"}.get(res["variant"], "?"),
+                       "l2": "inputs larger than L2: W (%.2f GB) streams from HBM every call" % (wl.V * wl.d * 2 / 1e9),
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "mean_accept_len": res["mean_accept"]},
+            "calls_per_s": world * K / (total_ms * 1e-3),
+            "median_ms_per_step": res["median_ms"],
+            "clocks": res["clocks"],
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": res["h2d"],
+                    "d2h_bytes_per_step": res["d2h"], "steps": res["e2e_steps"]},
+            "gpu_launches": res["launches"] * K,
+            "roofline": roofline_of(wl, peaks, res["mean_ms"], sustained=total_ms > 1000, which=which),
+            "cpu_baseline": cpu,
+            "other_workloads": others,
+        }
+        print(json.dumps(line), flush=True)
+    if args.dist:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,87 @@
+"""Parity at the published workload sizes, in the launch configuration the benchmark times
+(variant chosen automatically).  The CPU checker recomputes whole sequences; where a workload
+has several sequences a sample of them is checked."""
+import numpy as np
+import pytest
+
+import jd_testlib as T
+from paper_2501_19309_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None):
+    """cases: list of (mode, tau or None)."""
+    from paper_2501_19309_b200 import jd
+    wl = I.CONFIGS[cfg]
+    inp = I.make_inputs(wl, data_seed)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    rep = T.Report()
+    for mode, tau in cases:
+        tau = inp.tau if tau is None else tau
+        out = ver.verify(dev["H"], dev["x"], dev["dl"], tau, inp.seed, mode)
+        assert ver.device_status() == jd.JD_OK
+        if expect_variant:
+            assert ver.launch_info()[0] == jd.VARIANTS[expect_variant]
+        got = T.to_numpy(out)
+        ref = T.run_oracle(inp, mode, tau=tau, sequences=sequences)
+        T.compare(got, ref, mode, wl.M, rep)
+    ver.close()
+    del dev
+    import torch
+    torch.cuda.empty_cache()
+    print("\n%s: %s" % (wl.name, rep))
+    return rep, inp
+
+
+@pytest.mark.parametrize("data_seed", [0, 1])
+def test_cfg1_8b_head(data_seed):
+    cases = [("judge_or_standard", 0.3), ("judge_or_standard", 0.5), ("judge_or_standard", 0.7)]
+    if data_seed == 0:
+        cases += [("standard", None), ("judge", None)]
+    full_case(1, data_seed, cases, expect_variant="fused")
+
+
+def test_cfg2_70b_head_sampled_sequences():
+    rep, _ = full_case(2, 0, [("judge_or_standard", None)], sequences=[0, 3], expect_variant="fused")
+    assert rep.sequences == 2
+
+
+def test_cfg3_405b_head_forced_rejection():
+    from paper_2501_19309_b200 import jd
+    wl = I.CONFIGS[3]
+    inp = I.make_inputs(wl, 0)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    rep = T.Report()
+    for mode in ("standard", "judge", "judge_or_standard"):
+        out = ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau, inp.seed, mode)
+        assert ver.device_status() == jd.JD_OK and ver.launch_info()[0] == jd.JD_VARIANT_FUSED
+        got = T.to_numpy(out)
+        assert got["accept_len"][0] <= wl.forced_reject_at           # rejection forced at slot 12
+        assert got["masks"][0, wl.forced_reject_at] == 0
+        if mode == "judge_or_standard":                              # one full checker pass (the slow part)
+            ref = T.run_oracle(inp, mode)
+            T.compare(got, ref, mode, wl.M, rep)
+    ver.close()
+    print("\ncfg3:", rep)
+
+
+def test_cfg3_masks_independent_of_mode():
+    wl = I.CONFIGS[3].scaled("cfg3-narrow", d=1024)
+    inp = I.make_inputs(wl, 0)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    masks = [T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau, 0, m))["masks"]
+             for m in ("standard", "judge", "judge_or_standard")]
+    assert np.array_equal(masks[0], masks[1]) and np.array_equal(masks[0], masks[2])
+    for mode in ("standard", "judge"):
+        got = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau, 0, mode))
+        T.compare(got, T.run_oracle(inp, mode, seed=0), mode, wl.M)
+    ver.close()
+
+
+def test_cfg4_batched_sampled_sequences():
+    rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[0, 37, 63])
+    assert rep.sequences == 3

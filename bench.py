@@ -93,6 +93,20 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(values, device, dist_on: bool):
+    """Element-wise maximum of a few floats over all ranks (the slowest rank sets the time)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist_on:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_value(units_per_rank_step: int, steps: int, world: int, max_seconds: float) -> float:
+    """Whole-job throughput of independent replicas: all ranks' units over the slowest rank's time."""
+    return world * units_per_rank_step * steps / max_seconds
+
+
 def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, which: str) -> dict:
     bytes_alg = wl.V * wl.d * 2 + wl.R * wl.d * 2            # W once + H once
     flops = 2.0 * wl.R * wl.V * wl.d
@@ -281,14 +295,11 @@ def main() -> None:
     res = measure_workload(wl, args, torch, jd, device, data_seed=rank, sample_clocks=True)
 
     # max over ranks of the timed region, sum of the units
-    t = torch.tensor([res["total_ms"], res["e2e_s"]], dtype=torch.float64, device=device)
-    if args.dist:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    total_ms, e2e_s = float(t[0]), float(t[1])
+    total_ms, e2e_s = max_over_ranks([res["total_ms"], res["e2e_s"]], device, args.dist)
     K = args.steps
     tokens_per_step = wl.B * wl.M
-    value = world * tokens_per_step * K / (total_ms * 1e-3)
-    e2e_value = world * tokens_per_step * res["e2e_steps"] / e2e_s
+    value = aggregate_value(tokens_per_step, K, world, total_ms * 1e-3)
+    e2e_value = aggregate_value(tokens_per_step, res["e2e_steps"], world, e2e_s)
 
     others = {}
     if rank == 0 and args.others:

@@ -159,6 +159,28 @@ jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launche
 jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot,
                                const int32_t* stream, int32_t n, float* out, void* cuda_stream);
 
+/* Handle-free form of jd_verify for callers that must not allocate device memory when they
+ * verify: servers whose own pool already owns the whole device, decode loops that cannot afford
+ * the synchronisation an allocation implies, code barred from allocating after start-up.
+ * (The paper has no counterpart; this is a deployment convenience of this library.)
+ * It runs the fused tensor-core variant only: bf16, d % 64 == 0, B*(M+1) <= 96, and V small
+ * enough for that variant; anything else returns JD_ERR_UNSUPPORTED and launches nothing.
+ * The kernel's scratch (591,872 bytes) is a fixed array inside the library's device image: every
+ * GPU that loads the library holds it until the process exits. No cudaMalloc, cudaFree or other
+ * allocating call is made here.
+ *   d, V, W, w_judge, b_judge : the head, as for jd_set_head (device pointers, 16-byte aligned)
+ *   args                     : as for jd_verify (device pointers); variant must be AUTO or FUSED,
+ *                              logits_debug NULL
+ *   device_status            : optional device pointer to one uint32 that receives the call's
+ *                              device status (JD_OK, JD_ERR_TIMEOUT, JD_ERR_BAD_TOKEN); NULL to skip
+ * The call uses the CURRENT device. Its first call on a device looks up the array's device
+ * address and the SM count; make that first call outside any stream capture. All calls on a
+ * device share the one array, which keeps the previous call's contents (the words that must
+ * start at zero are cleared on the stream each time): calls that overlap on the GPU, from any
+ * stream or thread, race with each other, so order them. Asynchronous on `cuda_stream`. */
+jd_status_t jd_verify_static(int32_t d, int32_t V, const void* W, const void* w_judge, float b_judge,
+                             const jd_verify_args_t* args, uint32_t* device_status, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

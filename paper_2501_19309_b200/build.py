@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libjd_b200.so")
-SOURCES = ["jd_api.cu", "jd_simt.cu", "jd_fused_sm100.cu"]
+SOURCES = ["jd_api.cu", "jd_simt.cu", "jd_fused_sm100.cu", "jd_static.cu"]
 HEADERS = ["jd_common.cuh", "jd_kernels.h"]
 
 

@@ -29,7 +29,8 @@ RESAMPLE = {"residual": JD_RESAMPLE_RESIDUAL, "target_p": JD_RESAMPLE_TARGET_P}
 VARIANTS = {"auto": JD_VARIANT_AUTO, "simt": JD_VARIANT_SIMT, "fused": JD_VARIANT_FUSED, "batched": JD_VARIANT_BATCHED}
 
 EXPORTS = ["jd_version", "jd_status_string", "jd_workspace_bytes", "jd_create", "jd_destroy", "jd_set_head",
-           "jd_verify", "jd_verify_host", "jd_last_device_status", "jd_last_launch_info", "jd_philox_uniforms"]
+           "jd_verify", "jd_verify_host", "jd_last_device_status", "jd_last_launch_info", "jd_philox_uniforms",
+           "jd_verify_static"]
 
 
 class jd_config_t(C.Structure):
@@ -79,6 +80,8 @@ def load():
     lib.jd_last_launch_info.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     lib.jd_philox_uniforms.argtypes = [C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                        C.c_void_p]
+    lib.jd_verify_static.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_float,
+                                     C.POINTER(jd_verify_args_t), C.c_void_p, C.c_void_p]
     for name in EXPORTS:
         if name not in ("jd_version", "jd_status_string", "jd_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -142,6 +145,14 @@ def jd_philox_uniforms(seed: int, b_ptr: int, slot_ptr: int, stream_idx_ptr: int
     return load().jd_philox_uniforms(C.c_uint64(seed), C.c_void_p(b_ptr), C.c_void_p(slot_ptr),
                                      C.c_void_p(stream_idx_ptr), C.c_int32(n), C.c_void_p(out_ptr),
                                      C.c_void_p(stream_ptr))
+
+
+def jd_verify_static(d: int, V: int, W_ptr: int, w_judge_ptr: int, b_judge: float, args: jd_verify_args_t,
+                     device_status_ptr: int = 0, stream_ptr: int = 0) -> int:
+    """Handle-free verification that allocates nothing (fixed scratch inside the library); see jd.h."""
+    return load().jd_verify_static(C.c_int32(d), C.c_int32(V), C.c_void_p(W_ptr), C.c_void_p(w_judge_ptr),
+                                   C.c_float(b_judge), C.byref(args), C.c_void_p(device_status_ptr or None),
+                                   C.c_void_p(stream_ptr))
 
 
 # ------------------------------------------------------------------ tensor-level convenience

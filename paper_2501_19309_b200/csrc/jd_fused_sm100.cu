@@ -134,19 +134,23 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   uint32_t r[16];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      : "r"(taddr)
+      : "memory");
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ float tmem_ld1(uint32_t taddr) {
-  uint32_t r;
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-  return __uint_as_float(r);
+// issue only; the value is valid after tmem_wait_ld8 has been given the registers
+__device__ __forceinline__ void tmem_ld1_issue(uint32_t taddr, uint32_t& r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld8(uint32_t* r) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
+               :: "memory");
 }
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
@@ -203,10 +207,23 @@ __device__ __forceinline__ void load_chunk(int i, int c0, int n_ovf, uint32_t tm
     tmem_ld16(tmem_lane_base + (uint32_t)((i - n_ovf) * N_PAD + c0), v);
   }
 }
+// logits of row r in tiles i0 .. i0+7 (those below T) for this thread's lane, fetched together
 template <int N_PAD>
-__device__ __forceinline__ float load_one(int i, int r, int n_ovf, uint32_t tmem_lane_base, const float* ovf, int tid) {
-  if (i < n_ovf) return ovf[((size_t)i * N_PAD + r) * kVocabTile + tid];
-  return tmem_ld1(tmem_lane_base + (uint32_t)((i - n_ovf) * N_PAD + r));
+__device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, uint32_t tmem_lane_base, const float* ovf,
+                                           int tid, float* out) {
+  uint32_t raw[8];
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int i = i0 + u;
+    raw[u] = 0u;
+    if (i < T) {
+      if (i < n_ovf) raw[u] = __float_as_uint(ovf[((size_t)i * N_PAD + r) * kVocabTile + tid]);
+      else tmem_ld1_issue(tmem_lane_base + (uint32_t)((i - n_ovf) * N_PAD + r), raw[u]);
+    }
+  }
+  tmem_wait_ld8(raw);
+#pragma unroll
+  for (int u = 0; u < 8; ++u) out[u] = __uint_as_float(raw[u]);
 }
 
 template <int N_PAD>
@@ -359,13 +376,41 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
     // (b) while W streams: draft-row statistics over this CTA's vocabulary slice, judge dots
     const int v_lo = t0 * kVocabTile, v_hi = min(V, (t0 + T) * kVocabTile);
+    const bool vec4 = (V % 4) == 0;   // rows are 16-byte aligned only then
     for (int bm = warp; bm < BM; bm += 4) {
       const float* row = cp.draft_logits + (size_t)bm * V;
       float m = -INFINITY, s = 0.f;
-      for (int v = v_lo + lane; v < v_hi; v += 32) {
-        const float xv = __ldg(row + v);
-        if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
-        else if (xv != -INFINITY) s += __expf(xv - m);
+      if (vec4) {
+        // eight 128-entry tiles per pass: all loads of the pass are issued before any arithmetic
+        for (int i0 = 0; i0 < T; i0 += 8) {
+          float4 x[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int v = v_lo + (i0 + u) * kVocabTile + lane * 4;
+            x[u] = (i0 + u < T && v < V) ? __ldg(reinterpret_cast<const float4*>(row + v))
+                                         : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+          }
+          float mm = -INFINITY;
+#pragma unroll
+          for (int u = 0; u < 8; ++u) mm = fmaxf(mm, fmaxf(fmaxf(x[u].x, x[u].y), fmaxf(x[u].z, x[u].w)));
+          const float mn = fmaxf(m, mm);
+          if (mn == -INFINITY) continue;
+          float acc = 0.f;
+          const float off = mn * kLog2e;
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            acc += exp2f(fmaf(x[u].x, kLog2e, -off)) + exp2f(fmaf(x[u].y, kLog2e, -off));
+            acc += exp2f(fmaf(x[u].z, kLog2e, -off)) + exp2f(fmaf(x[u].w, kLog2e, -off));
+          }
+          s = s * __expf(m - mn) + acc;
+          m = mn;
+        }
+      } else {
+        for (int v = v_lo + lane; v < v_hi; v += 32) {
+          const float xv = __ldg(row + v);
+          if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
+          else if (xv != -INFINITY) s += __expf(xv - m);
+        }
       }
       ms_warp_reduce(m, s);
       if (lane == 0) {
@@ -529,14 +574,23 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
         const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;   // used only when kind == 0
         double sr = 0.0, sp = 0.0;
-        for (int i = 0; i < T; ++i) {
-          const int vg = (t0 + i) * kVocabTile + tid;
-          const float logit = load_one<N_PAD>(i, row, n_ovf, tmem_lane_base, ovf, tid);
-          if (vg < V) {
-            float p, r;
-            sample_weights(logit, lse_p, kind, kind == 0 ? __ldg(dlrow + vg) : 0.f, lse_q, p, r);
-            sr += (double)r;
-            sp += (double)p;
+        for (int i0 = 0; i0 < T; i0 += 8) {
+          float dv[8], lg[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int vg = (t0 + i0 + u) * kVocabTile + tid;
+            dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
+          }
+          load_cols8<N_PAD>(i0, T, row, n_ovf, tmem_lane_base, ovf, tid, lg);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int vg = (t0 + i0 + u) * kVocabTile + tid;
+            if (i0 + u < T && vg < V) {
+              float p, r;
+              sample_weights(lg[u], lse_p, kind, dv[u], lse_q, p, r);
+              sr += (double)r;
+              sp += (double)p;
+            }
           }
         }
         sr = warp_sum_double(sr);
@@ -623,7 +677,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         int token = -1, last_token = -1;
         for (int i = 0; i < T && token < 0; ++i) {
           const int vg = (t0 + i) * kVocabTile + tid;
-          const float logit = load_one<N_PAD>(i, row, n_ovf, tmem_lane_base, ovf, tid);
+          float lgv[8];
+          load_cols8<N_PAD>(i, min(T, i + 1), row, n_ovf, tmem_lane_base, ovf, tid, lgv);
+          const float logit = lgv[0];
           float p = 0.f, r = 0.f;
           if (vg < V) sample_weights(logit, lse_p, kind, kind == 0 ? __ldg(dlrow + vg) : 0.f, lse_q, p, r);
           // ordered inclusive scan over the 128 lanes of the tile, in double

@@ -165,7 +165,7 @@ jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* s
  * (The paper has no counterpart; this is a deployment convenience of this library.)
  * It runs the fused tensor-core variant only: bf16, d % 64 == 0, B*(M+1) <= 96, and V small
  * enough for that variant; anything else returns JD_ERR_UNSUPPORTED and launches nothing.
- * The kernel's scratch (591,872 bytes) is a fixed array inside the library's device image: every
+ * The kernel's scratch (592,896 bytes) is a fixed array inside the library's device image: every
  * GPU that loads the library holds it until the process exits. No cudaMalloc, cudaFree or other
  * allocating call is made here.
  *   d, V, W, w_judge, b_judge : the head, as for jd_set_head (device pointers, 16-byte aligned)

@@ -36,7 +36,7 @@ constexpr int kEpiThreads = 128;
 constexpr int kBlockK = 64;                      // bf16 elements per k-slice = one 128-byte swizzle row
 constexpr int kWStageBytes = kVocabTile * 128;   // 16 KB
 constexpr int kTmemCols = 512;
-constexpr int kMiscBytes = 8192;                 // barriers + reduction scratch at the head of smem
+constexpr int kMiscBytes = 13312;                // barriers + reduction scratch at the head of smem
 constexpr int kMaxStages = 12;
 constexpr int kHStages = 4;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -179,33 +179,82 @@ struct Misc {
   uint64_t drained;
   uint32_t tmem_base;
   int abort_flag;
+  int glist_n;              // rows whose drafted token lies in this CTA's vocabulary slice
   float wmax[4][N_PAD];
   float wsum[4][N_PAD];
   float cta_max[N_PAD];
-  float lse[N_PAD];       // log-normaliser of every row (all CTAs compute the same values)
-  float rmax[N_PAD];
+  float lse[N_PAD];         // log-normaliser of every row
   float qlse[N_PAD];
-  int x_row[N_PAD];       // drafted token of row r (rows j < M), -1 otherwise
-  int sel_row[N_PAD];
-  int sel_kind[N_PAD];
-  float sel_lse_p[N_PAD];
-  float sel_lse_q[N_PAD];
-  float sel_u[N_PAD];
-  double wd[2][4];
+  int x_row[N_PAD];         // drafted token of row r (rows j < M), -1 otherwise
+  int glist[N_PAD];
+  // per sequence (B <= N_PAD / 2 because M >= 1)
+  int sel_row[N_PAD / 2];
+  int sel_kind[N_PAD / 2];
+  float sel_lse_p[N_PAD / 2];
+  float sel_lse_q[N_PAD / 2];
+  float sel_u[N_PAD / 2];
+  double wd_r[N_PAD / 2][4];
+  double wd_p[N_PAD / 2][4];
+  int own_cta[N_PAD / 2];
+  int own_usep[N_PAD / 2];
+  double own_prefix[N_PAD / 2];
+  double own_T[N_PAD / 2];
+  double tsum[4][8];
+  double wscan[4];
   int cand[4];
   int lastpos[4];
 };
 
-// logit of (tile i, this thread's lane, row r): from TMEM or from the overflow copy in smem
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+// one wait for two 16-column loads; the registers pass through the statement so that nothing
+// that consumes them can be scheduled ahead of the wait
+__device__ __forceinline__ void tmem_wait_ld32(uint32_t* a, uint32_t* b) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+                 "+r"(a[8]), "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]),
+                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
+                 "+r"(b[8]), "+r"(b[9]), "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15])
+               :: "memory");
+}
+
+// logits of rows c0..c0+15 for this thread's lane in tiles i0 and i0+1 (zeros past T): from TMEM,
+// or from the overflow copy in shared memory
 template <int N_PAD>
-__device__ __forceinline__ void load_chunk(int i, int c0, int n_ovf, uint32_t tmem_lane_base, const float* ovf, int tid,
-                                           float* v) {
-  if (i < n_ovf) {
+__device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, uint32_t tmem_lane_base, const float* ovf,
+                                            int tid, float* v0, float* v1) {
+  uint32_t a[16], b[16];
 #pragma unroll
-    for (int k = 0; k < 16; ++k) v[k] = ovf[((size_t)i * N_PAD + c0 + k) * kVocabTile + tid];
+  for (int k = 0; k < 16; ++k) { a[k] = 0u; b[k] = 0u; }
+  if (i0 < n_ovf) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) a[k] = __float_as_uint(ovf[((size_t)i0 * N_PAD + c0 + k) * kVocabTile + tid]);
   } else {
-    tmem_ld16(tmem_lane_base + (uint32_t)((i - n_ovf) * N_PAD + c0), v);
+    tmem_ld16_issue(tmem_lane_base + (uint32_t)((i0 - n_ovf) * N_PAD + c0), a);
   }
+  if (i0 + 1 < T) {
+    if (i0 + 1 < n_ovf) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) b[k] = __float_as_uint(ovf[((size_t)(i0 + 1) * N_PAD + c0 + k) * kVocabTile + tid]);
+    } else {
+      tmem_ld16_issue(tmem_lane_base + (uint32_t)((i0 + 1 - n_ovf) * N_PAD + c0), b);
+    }
+  }
+  tmem_wait_ld32(a, b);
+#pragma unroll
+  for (int k = 0; k < 16; ++k) { v0[k] = __uint_as_float(a[k]); v1[k] = __uint_as_float(b[k]); }
 }
 // logits of row r in tiles i0 .. i0+7 (those below T) for this thread's lane, fetched together
 template <int N_PAD>
@@ -224,6 +273,42 @@ __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, uint
   tmem_wait_ld8(raw);
 #pragma unroll
   for (int u = 0; u < 8; ++u) out[u] = __uint_as_float(raw[u]);
+}
+
+// Reduces 16 per-lane values over the 32 lanes of a warp with 16 shuffles instead of 80: every
+// step halves the number of values a lane keeps. On return lane l holds the reduction of value
+// index reduce16_index(l) (lanes 2j and 2j+1 hold the same one).
+template <bool kMax>
+__device__ __forceinline__ float warp_reduce16(const float* v, int lane) {
+  auto op = [](float x, float y) { return kMax ? fmaxf(x, y) : x + y; };
+  float a[8], b4[4], c2[2];
+  const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4, h2 = lane & 2;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const float send = h16 ? v[k] : v[k + 8];
+    const float keep = h16 ? v[k + 8] : v[k];
+    a[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 16));
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const float send = h8 ? a[k] : a[k + 4];
+    const float keep = h8 ? a[k + 4] : a[k];
+    b4[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 8));
+  }
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const float send = h4 ? b4[k] : b4[k + 2];
+    const float keep = h4 ? b4[k + 2] : b4[k];
+    c2[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 4));
+  }
+  const float send = h2 ? c2[0] : c2[1];
+  const float keep = h2 ? c2[1] : c2[0];
+  float d = op(keep, __shfl_xor_sync(0xffffffffu, send, 2));
+  d = op(d, __shfl_xor_sync(0xffffffffu, d, 1));
+  return d;
+}
+__device__ __forceinline__ int reduce16_index(int lane) {
+  return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
 }
 
 template <int N_PAD>
@@ -259,6 +344,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     mbar_init(smem_u32(&ms.acc_full[1]), 1);
     mbar_init(smem_u32(&ms.drained), 1);
     ms.abort_flag = 0;
+    ms.glist_n = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < N_PAD) {
@@ -281,6 +367,10 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = ms.tmem_base;
+  if (tid < R) {   // rows whose drafted token this CTA's slice holds (usually none or one)
+    const int x = ms.x_row[tid];
+    if (x >= t0 * kVocabTile && x < (t0 + T) * kVocabTile) ms.glist[atomicAdd(&ms.glist_n, 1)] = tid;
+  }
 
   // group 0 = the n_ovf overflow tiles (if any), group 1 = the TMEM-resident tiles
   const int g_begin[2] = {0, n_ovf};
@@ -448,66 +538,69 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     epi_sync();
     ok = ok && (*abort_flag == 0);
 
-    // (d) per-row max over this CTA's slice, and the gather of the drafted tokens' logits
-    {
-      float m[N_PAD];
+    // (d) gather of the drafted tokens' logits (rows listed in the prologue), per-row max
+    if (ok) {
+      const int ng = ms.glist_n;
+      for (int e = 0; e < ng; ++e) {
+        const int r = ms.glist[e], x = ms.x_row[r];
+        const int i = x / kVocabTile - t0;
+        float one[8];
+        load_cols8<N_PAD>(i, i + 1, r, n_ovf, tmem_lane_base, ovf, tid, one);
+        if (tid == (x % kVocabTile)) ws.gath[r] = one[0];
+      }
+    }
 #pragma unroll
-      for (int r = 0; r < N_PAD; ++r) m[r] = -INFINITY;
+    for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+      float mx[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) mx[k] = -INFINITY;
       if (ok) {
-        for (int i = 0; i < T; ++i) {
-          const int vg = (t0 + i) * kVocabTile + tid;
-          const bool valid = vg < V;
+        for (int i0 = 0; i0 < T; i0 += 2) {
+          float v0[16], v1[16];
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, tmem_lane_base, ovf, tid, v0, v1);
+          const bool val0 = (t0 + i0) * kVocabTile + tid < V;
+          const bool val1 = (i0 + 1 < T) && ((t0 + i0 + 1) * kVocabTile + tid < V);
+          if (val0) {
 #pragma unroll
-          for (int c0 = 0; c0 < N_PAD; c0 += 16) {
-            float v[16];
-            load_chunk<N_PAD>(i, c0, n_ovf, tmem_lane_base, ovf, tid, v);
+            for (int k = 0; k < 16; ++k) mx[k] = fmaxf(mx[k], v0[k]);
+          }
+          if (val1) {
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
-              if (valid) {
-                m[c0 + k] = fmaxf(m[c0 + k], v[k]);
-                if (ms.x_row[c0 + k] == vg) ws.gath[c0 + k] = v[k];
-              }
-            }
+            for (int k = 0; k < 16; ++k) mx[k] = fmaxf(mx[k], v1[k]);
           }
         }
       }
-#pragma unroll
-      for (int r = 0; r < N_PAD; ++r) {
-        float x = m[r];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
-        if (lane == 0) ms.wmax[warp][r] = x;
-      }
+      const float red = warp_reduce16<true>(mx, lane);
+      if ((lane & 1) == 0) ms.wmax[warp][c0 + reduce16_index(lane)] = red;
     }
     epi_sync();
     if (tid < N_PAD) ms.cta_max[tid] = fmaxf(fmaxf(ms.wmax[0][tid], ms.wmax[1][tid]), fmaxf(ms.wmax[2][tid], ms.wmax[3][tid]));
     epi_sync();
 
     // (e) per-row sum exp(L - cta max)
-    {
-      float s[N_PAD];
 #pragma unroll
-      for (int r = 0; r < N_PAD; ++r) s[r] = 0.f;
+    for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+      float acc[16], cm[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) { acc[k] = 0.f; cm[k] = ms.cta_max[c0 + k] * kLog2e; }
       if (ok) {
-        for (int i = 0; i < T; ++i) {
-          const bool valid = (t0 + i) * kVocabTile + tid < V;
+        for (int i0 = 0; i0 < T; i0 += 2) {
+          float v0[16], v1[16];
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, tmem_lane_base, ovf, tid, v0, v1);
+          const bool val0 = (t0 + i0) * kVocabTile + tid < V;
+          const bool val1 = (i0 + 1 < T) && ((t0 + i0 + 1) * kVocabTile + tid < V);
+          if (val0) {
 #pragma unroll
-          for (int c0 = 0; c0 < N_PAD; c0 += 16) {
-            float v[16];
-            load_chunk<N_PAD>(i, c0, n_ovf, tmem_lane_base, ovf, tid, v);
+            for (int k = 0; k < 16; ++k) acc[k] += fast_exp2(fmaf(v0[k], kLog2e, -cm[k]));
+          }
+          if (val1) {
 #pragma unroll
-            for (int k = 0; k < 16; ++k)
-              if (valid) s[c0 + k] += exp2f((v[k] - ms.cta_max[c0 + k]) * kLog2e);
+            for (int k = 0; k < 16; ++k) acc[k] += fast_exp2(fmaf(v1[k], kLog2e, -cm[k]));
           }
         }
       }
-#pragma unroll
-      for (int r = 0; r < N_PAD; ++r) {
-        float x = s[r];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-        if (lane == 0) ms.wsum[warp][r] = x;
-      }
+      const float red = warp_reduce16<false>(acc, lane);
+      if ((lane & 1) == 0) ms.wsum[warp][c0 + reduce16_index(lane)] = red;
     }
     epi_sync();
     if (tid < R) {
@@ -527,34 +620,63 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     epi_sync();
     ok = (*abort_flag == 0);
 
+    // (f) fold the per-CTA statistics: the R target rows and the B*M draft rows are dealt out
+    // over the grid, one per warp, so that no CTA reads more than a few rows' worth of partials
     if (ok) {
-      // (f) fold the per-CTA statistics of every row (every CTA computes the same numbers)
-      for (int r = warp; r < R; r += 4) {
-        float m = -INFINITY, s = 0.f;
-        for (int c = lane; c < G; c += 32)
-          ms_combine(m, s, __ldcg(ws.part_max + (size_t)r * G + c), __ldcg(ws.part_sum + (size_t)r * G + c));
-        ms_warp_reduce(m, s);
+      for (int it = cta + G * warp; it < R + BM; it += 4 * G) {
+        const bool is_p = it < R;
+        const float* pm = is_p ? ws.part_max + (size_t)it * G : ws.qpart_max + (size_t)(it - R) * G;
+        const float* ps = is_p ? ws.part_sum + (size_t)it * G : ws.qpart_sum + (size_t)(it - R) * G;
+        float vm[8], vs[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int c = lane + 32 * u;
+          vm[u] = c < G ? __ldcg(pm + c) : -INFINITY;
+          vs[u] = c < G ? __ldcg(ps + c) : 0.f;
+        }
+        float m = vm[0];
+#pragma unroll
+        for (int u = 1; u < 8; ++u) m = fmaxf(m, vm[u]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        float sacc = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (vs[u] > 0.f) sacc += vs[u] * fast_exp2((vm[u] - m) * kLog2e);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, o);
         if (lane == 0) {
-          const float lse = m + logf(s);
-          ms.rmax[r] = m;
-          ms.lse[r] = lse;
-          if (cta == 0) {
-            if (cp.row_max_out) cp.row_max_out[r] = m;
-            if (cp.row_lse_out) cp.row_lse_out[r] = lse;
+          const float lse = m + logf(sacc);
+          if (is_p) {
+            ws.row_lse[it] = lse;
+            if (cp.row_max_out) cp.row_max_out[it] = m;
+            if (cp.row_lse_out) cp.row_lse_out[it] = lse;
+          } else {
+            ws.q_lse[it - R] = lse;
           }
         }
       }
-      for (int bm = warp; bm < BM; bm += 4) {
-        float m = -INFINITY, s = 0.f;
-        for (int c = lane; c < G; c += 32)
-          ms_combine(m, s, __ldcg(ws.qpart_max + (size_t)bm * G + c), __ldcg(ws.qpart_sum + (size_t)bm * G + c));
-        ms_warp_reduce(m, s);
-        if (lane == 0) ms.qlse[bm] = m + logf(s);
+    }
+    __threadfence();
+    epi_sync();
+
+    // ------------------------------------------------------------------ grid barrier 2
+    if (tid == 0) {
+      if (!ok || !grid_arrive_and_wait(ws.barrier + 1, (unsigned)G, abort_flag)) {
+        *abort_flag = 1;
+        set_status(ws.status, JD_ERR_TIMEOUT);
       }
     }
     epi_sync();
+    ok = (*abort_flag == 0);
     if (ok) {
-      // (g) tests, mask, accepted prefix (Eq. 4; Sec. 4.1): one warp per sequence
+      if (tid < R) ms.lse[tid] = __ldcg(ws.row_lse + tid);
+      if (tid < BM) ms.qlse[tid] = __ldcg(ws.q_lse + tid);
+    }
+    epi_sync();
+    if (ok) {
+      // (g) tests, mask, accepted prefix (Eq. 4; Sec. 4.1): one warp per sequence, identical in
+      // every CTA; CTA 0 writes the outputs
       Workspace lw = ws;
       lw.row_lse = ms.lse;
       lw.q_lse = ms.qlse;
@@ -595,21 +717,20 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
         sr = warp_sum_double(sr);
         sp = warp_sum_double(sp);
-        if (lane == 0) { ms.wd[0][warp] = sr; ms.wd[1][warp] = sp; }
-        epi_sync();
-        if (tid == 0) {
-          ws.mass_r[(size_t)b * G + cta] = (ms.wd[0][0] + ms.wd[0][1]) + (ms.wd[0][2] + ms.wd[0][3]);
-          ws.mass_p[(size_t)b * G + cta] = (ms.wd[1][0] + ms.wd[1][1]) + (ms.wd[1][2] + ms.wd[1][3]);
-        }
-        epi_sync();
+        if (lane == 0) { ms.wd_r[b][warp] = sr; ms.wd_p[b][warp] = sp; }
       }
+    }
+    epi_sync();
+    if (ok && tid < cp.B) {
+      ws.mass_r[(size_t)tid * G + cta] = (ms.wd_r[tid][0] + ms.wd_r[tid][1]) + (ms.wd_r[tid][2] + ms.wd_r[tid][3]);
+      ws.mass_p[(size_t)tid * G + cta] = (ms.wd_p[tid][0] + ms.wd_p[tid][1]) + (ms.wd_p[tid][2] + ms.wd_p[tid][3]);
     }
     __threadfence();
     epi_sync();
 
-    // ------------------------------------------------------------------ grid barrier 2
+    // ------------------------------------------------------------------ grid barrier 3
     if (tid == 0) {
-      if (!ok || !grid_arrive_and_wait(ws.barrier + 1, (unsigned)G, abort_flag)) {
+      if (!ok || !grid_arrive_and_wait(ws.barrier + 2, (unsigned)G, abort_flag)) {
         *abort_flag = 1;
         set_status(ws.status, JD_ERR_TIMEOUT);
       }
@@ -617,23 +738,34 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     epi_sync();
     ok = (*abort_flag == 0);
 
-    // (i) inverse CDF in ascending token id: find the owning CTA, then the token inside it
+    // (i) inverse CDF in ascending token id. First, one warp per sequence finds the CTA whose
+    // slice contains T = u * total (same arithmetic in every CTA, so every CTA agrees) ...
     if (ok) {
-      for (int b = 0; b < cp.B; ++b) {
-        // every warp scans the per-CTA masses in the same order: lane l owns CTAs [l*per, (l+1)*per)
-        const int per = (G + 31) / 32;
+      const int per = (G + 31) / 32;   // lane l owns CTAs [l*per, (l+1)*per), per <= 8
+      for (int b = warp; b < cp.B; b += 4) {
         const double* mass = ws.mass_r + (size_t)b * G;
-        bool use_p = false;
+        double mc[8];
         double chunk = 0.0;
-        for (int c = lane * per; c < min(G, (lane + 1) * per); ++c) chunk += __ldcg(mass + c);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int c = lane * per + u;
+          mc[u] = (u < per && c < G) ? __ldcg(mass + c) : 0.0;
+          chunk += mc[u];
+        }
         double total = warp_sum_double(chunk);
+        int use_p = 0;
         if (!(total > 0.0)) {   // identically zero residual: draw from p
-          use_p = true;
+          use_p = 1;
           mass = ws.mass_p + (size_t)b * G;
           chunk = 0.0;
-          for (int c = lane * per; c < min(G, (lane + 1) * per); ++c) chunk += __ldcg(mass + c);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int c = lane * per + u;
+            mc[u] = (u < per && c < G) ? __ldcg(mass + c) : 0.0;
+            chunk += mc[u];
+          }
         }
-        // exclusive prefix of the lane chunks (sequential over lanes, identical in every warp)
+        // exclusive prefix of the lane chunks, summed in lane order
         double excl = 0.0, run = 0.0;
         for (int l = 0; l < 32; ++l) {
           const double cl = __shfl_sync(0xffffffffu, chunk, l);
@@ -642,16 +774,18 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
         total = run;
         const double Tt = (double)ms.sel_u[b] * total;
-        // owner = first CTA whose inclusive prefix exceeds T, else the last CTA with mass
         int owner = -1, last_mass = -1;
-        double my_prefix = 0.0;   // exclusive prefix of the owner, valid in the lane that finds it
+        double my_prefix = 0.0;
         {
           double c = excl;
-          for (int cc = lane * per; cc < min(G, (lane + 1) * per); ++cc) {
-            const double mc = __ldcg(mass + cc);
-            if (mc > 0.0) last_mass = cc;
-            if (owner < 0 && c + mc > Tt) { owner = cc; my_prefix = c; }
-            c += mc;
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int cc = lane * per + u;
+            if (u < per && cc < G) {
+              if (mc[u] > 0.0) last_mass = cc;
+              if (owner < 0 && c + mc[u] > Tt) { owner = cc; my_prefix = c; }
+              c += mc[u];
+            }
           }
         }
         const unsigned found = __ballot_sync(0xffffffffu, owner >= 0);
@@ -660,53 +794,94 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           const int src = __ffs(found) - 1;
           owner = __shfl_sync(0xffffffffu, owner, src);
           owner_prefix = __shfl_sync(0xffffffffu, my_prefix, src);
-        } else {
+        } else {   // T at or beyond the total after rounding: the last CTA that carries mass
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) last_mass = max(last_mass, __shfl_xor_sync(0xffffffffu, last_mass, o));
           owner = last_mass;
-          owner_prefix = -1.0;   // marks the "T beyond the total" fallback
+          owner_prefix = -1.0;
         }
-        if (owner != cta) continue;   // uniform over the CTA: every warp computed the same owner
-
+        if (lane == 0) {
+          ms.own_cta[b] = owner;
+          ms.own_prefix[b] = owner_prefix;
+          ms.own_T[b] = Tt;
+          ms.own_usep[b] = use_p;
+        }
+      }
+    }
+    epi_sync();
+    // ... then the owning CTA finds the tile from the tile masses and the token inside that tile
+    if (ok) {
+      for (int b = 0; b < cp.B; ++b) {
+        if (ms.own_cta[b] != cta) continue;
         const int row = ms.sel_row[b];
-        const int kind = use_p ? 1 : ms.sel_kind[b];
+        const int kind = ms.own_usep[b] ? 1 : ms.sel_kind[b];
         const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
         const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;
-        const bool beyond = owner_prefix < 0.0;
-        double c_tile = beyond ? 0.0 : owner_prefix;
+        const double Tt = ms.own_T[b];
+        const bool beyond = ms.own_prefix[b] < 0.0;
+        double c_run = beyond ? 0.0 : ms.own_prefix[b];
         int token = -1, last_token = -1;
-        for (int i = 0; i < T && token < 0; ++i) {
-          const int vg = (t0 + i) * kVocabTile + tid;
-          float lgv[8];
-          load_cols8<N_PAD>(i, min(T, i + 1), row, n_ovf, tmem_lane_base, ovf, tid, lgv);
-          const float logit = lgv[0];
-          float p = 0.f, r = 0.f;
-          if (vg < V) sample_weights(logit, lse_p, kind, kind == 0 ? __ldg(dlrow + vg) : 0.f, lse_q, p, r);
-          // ordered inclusive scan over the 128 lanes of the tile, in double
-          double incl = (double)r;
+        for (int i0 = 0; i0 < T && token < 0; i0 += 8) {
+          float dv[8], lg[8], rw[8];
 #pragma unroll
-          for (int o = 1; o < 32; o <<= 1) {
-            const double up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
+          for (int u = 0; u < 8; ++u) {
+            const int vg = (t0 + i0 + u) * kVocabTile + tid;
+            dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
           }
-          if (lane == 31) ms.wd[0][warp] = incl;
-          const unsigned pos = __ballot_sync(0xffffffffu, r > 0.f);
-          if (lane == 0) ms.lastpos[warp] = pos ? (31 - __clz(pos)) : -1;
-          epi_sync();
-          double off = c_tile;
-          for (int w = 0; w < warp; ++w) off += ms.wd[0][w];
-          const double tile_total = (ms.wd[0][0] + ms.wd[0][1]) + (ms.wd[0][2] + ms.wd[0][3]);
-          const unsigned hit = beyond ? 0u : __ballot_sync(0xffffffffu, off + incl > Tt);
-          if (lane == 0) ms.cand[warp] = hit ? (__ffs(hit) - 1) : -1;
-          epi_sync();
-          for (int w = 0; w < 4; ++w) {
-            if (token < 0 && ms.cand[w] >= 0) token = (t0 + i) * kVocabTile + w * 32 + ms.cand[w];
-            if (ms.lastpos[w] >= 0) last_token = (t0 + i) * kVocabTile + w * 32 + ms.lastpos[w];
+          load_cols8<N_PAD>(i0, T, row, n_ovf, tmem_lane_base, ovf, tid, lg);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int vg = (t0 + i0 + u) * kVocabTile + tid;
+            float p = 0.f, r = 0.f;
+            if (i0 + u < T && vg < V) sample_weights(lg[u], lse_p, kind, dv[u], lse_q, p, r);
+            rw[u] = r;
+            const double su = warp_sum_double((double)r);
+            if (lane == 0) ms.tsum[warp][u] = su;
           }
-          c_tile += tile_total;
+          epi_sync();
+          // the tile that contains T, else the last tile of this pass that carries mass
+          int ustar = -1, ulast = -1;
+          double c_before = c_run;
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const double tt = (ms.tsum[0][u] + ms.tsum[1][u]) + (ms.tsum[2][u] + ms.tsum[3][u]);
+            if (tt > 0.0) ulast = u;
+            if (ustar < 0) {
+              if (!beyond && c_run + tt > Tt) { ustar = u; c_before = c_run; }
+              c_run += tt;
+            }
+          }
+          const int usel = ustar >= 0 ? ustar : ulast;
+          if (usel >= 0) {
+            float r = 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) if (u == usel) r = rw[u];
+            double incl = (double)r;   // ordered inclusive scan over the 128 lanes of the tile
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+              const double up = __shfl_up_sync(0xffffffffu, incl, o);
+              if (lane >= o) incl += up;
+            }
+            if (lane == 31) ms.wscan[warp] = incl;
+            const unsigned pos = __ballot_sync(0xffffffffu, r > 0.f);
+            if (lane == 0) ms.lastpos[warp] = pos ? (31 - __clz(pos)) : -1;
+            epi_sync();
+            double off = c_before;
+            for (int w = 0; w < warp; ++w) off += ms.wscan[w];
+            const unsigned hit = (ustar >= 0) ? __ballot_sync(0xffffffffu, off + incl > Tt) : 0u;
+            if (lane == 0) ms.cand[warp] = hit ? (__ffs(hit) - 1) : -1;
+            epi_sync();
+            const int tile_v0 = (t0 + i0 + usel) * kVocabTile;
+            for (int w = 0; w < 4; ++w) {
+              if (token < 0 && ms.cand[w] >= 0) token = tile_v0 + w * 32 + ms.cand[w];
+              if (ms.lastpos[w] >= 0) last_token = tile_v0 + w * 32 + ms.lastpos[w];
+            }
+            // summation-order rounding can leave the tile without a hit: its last token with mass
+            if (ustar >= 0 && token < 0) token = last_token;
+          }
           epi_sync();
         }
-        if (token < 0) token = last_token;   // rounding at the upper edge: the last token with mass
+        if (token < 0) token = last_token;   // T beyond the total: the last token that carries mass
         if (tid == 0) cp.next_token[b] = token < 0 ? 0 : token;
       }
     }

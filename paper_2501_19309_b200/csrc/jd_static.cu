@@ -6,7 +6,7 @@
 // allocation would add an implicit device synchronisation, and code running under a policy
 // that forbids allocation after initialisation. jd_create allocates a workspace, so it is not
 // for them. This entry point needs no handle: the scratch memory of the fused kernel (per-CTA
-// softmax partials, gathered logits, per-CTA sampling masses, status word, grid-barrier
+// softmax partials, gathered logits, row normalisers, per-CTA sampling masses, status word, grid-barrier
 // counters) lives in a fixed array in the library's device image, which every GPU that loads
 // the library holds until the process exits.
 #include <cuda.h>
@@ -25,8 +25,9 @@ constexpr int kStaticMaxSeqs = kStaticMaxRows / 2;       // M >= 1, so B <= 48
 constexpr size_t kRowPartials = (size_t)kStaticMaxRows * kMaxCtas * sizeof(float);    //  98,304 B
 constexpr size_t kSeqMasses = (size_t)kStaticMaxSeqs * kMaxCtas * sizeof(double);     //  98,304 B
 constexpr size_t kSmall = 512;                           // 96 floats, rounded to 256-byte units
-// part_max, part_sum, qpart_max, qpart_sum | mass_r, mass_p | gath, qgath, judge_logit | status+barrier
-constexpr size_t kStaticScratchBytes = 4 * kRowPartials + 2 * kSeqMasses + 3 * kSmall + 512;   // 591,872 B
+// part_max, part_sum, qpart_max, qpart_sum | mass_r, mass_p | gath, qgath, judge_logit, row_lse, q_lse |
+// status + barrier counters
+constexpr size_t kStaticScratchBytes = 4 * kRowPartials + 2 * kSeqMasses + 5 * kSmall + 512;   // 592,896 B
 
 // The scratch itself. In host code this name is only a handle for cudaGetSymbolAddress; it is
 // not a device address and must never be passed to a kernel as is.
@@ -116,6 +117,8 @@ extern "C" jd_status_t jd_verify_static(int32_t d, int32_t V, const void* W, con
   ws.gath = (float*)take(kSmall);
   ws.qgath = (float*)take(kSmall);
   ws.judge_logit = (float*)take(kSmall);
+  ws.row_lse = (float*)take(kSmall);
+  ws.q_lse = (float*)take(kSmall);
   unsigned* own_status = (unsigned*)take(256);
   ws.status = device_status ? device_status : own_status;   // the caller's word receives the status if given
   ws.barrier = (unsigned*)take(256);

@@ -46,6 +46,7 @@ struct FusedParams {
   int num_tiles;    // ceil(V / 128)
   int stages;       // W ring depth
   int tmem_tiles;   // tiles resident in TMEM
+  int tile_stride;  // TMEM columns between consecutive tiles (>= rows, multiple of 8, <= N_PAD)
   int R;            // B * (M + 1)
   uint32_t off_h;   // byte offsets inside dynamic smem (from the 1024-aligned base)
   uint32_t off_ovf;
@@ -233,8 +234,8 @@ __device__ __forceinline__ void tmem_wait_ld32(uint32_t* a, uint32_t* b) {
 // logits of rows c0..c0+15 for this thread's lane in tiles i0 and i0+1 (zeros past T): from TMEM,
 // or from the overflow copy in shared memory
 template <int N_PAD>
-__device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, uint32_t tmem_lane_base, const float* ovf,
-                                            int tid, float* v0, float* v1) {
+__device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, int ts, uint32_t tmem_lane_base,
+                                            const float* ovf, int tid, float* v0, float* v1) {
   uint32_t a[16], b[16];
 #pragma unroll
   for (int k = 0; k < 16; ++k) { a[k] = 0u; b[k] = 0u; }
@@ -242,14 +243,14 @@ __device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, ui
 #pragma unroll
     for (int k = 0; k < 16; ++k) a[k] = __float_as_uint(ovf[((size_t)i0 * N_PAD + c0 + k) * kVocabTile + tid]);
   } else {
-    tmem_ld16_issue(tmem_lane_base + (uint32_t)((i0 - n_ovf) * N_PAD + c0), a);
+    tmem_ld16_issue(tmem_lane_base + (uint32_t)((i0 - n_ovf) * ts + c0), a);
   }
   if (i0 + 1 < T) {
     if (i0 + 1 < n_ovf) {
 #pragma unroll
       for (int k = 0; k < 16; ++k) b[k] = __float_as_uint(ovf[((size_t)(i0 + 1) * N_PAD + c0 + k) * kVocabTile + tid]);
     } else {
-      tmem_ld16_issue(tmem_lane_base + (uint32_t)((i0 + 1 - n_ovf) * N_PAD + c0), b);
+      tmem_ld16_issue(tmem_lane_base + (uint32_t)((i0 + 1 - n_ovf) * ts + c0), b);
     }
   }
   tmem_wait_ld32(a, b);
@@ -258,8 +259,8 @@ __device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, ui
 }
 // logits of row r in tiles i0 .. i0+7 (those below T) for this thread's lane, fetched together
 template <int N_PAD>
-__device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, uint32_t tmem_lane_base, const float* ovf,
-                                           int tid, float* out) {
+__device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, int ts, uint32_t tmem_lane_base,
+                                           const float* ovf, int tid, float* out) {
   uint32_t raw[8];
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
@@ -267,7 +268,7 @@ __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, uint
     raw[u] = 0u;
     if (i < T) {
       if (i < n_ovf) raw[u] = __float_as_uint(ovf[((size_t)i * N_PAD + r) * kVocabTile + tid]);
-      else tmem_ld1_issue(tmem_lane_base + (uint32_t)((i - n_ovf) * N_PAD + r), raw[u]);
+      else tmem_ld1_issue(tmem_lane_base + (uint32_t)((i - n_ovf) * ts + r), raw[u]);
     }
   }
   tmem_wait_ld8(raw);
@@ -423,7 +424,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           if (!ok) break;
           tc_fence_after();
           const uint32_t wb = sW + ws_i * kWStageBytes;
-          const uint32_t dcol = tmem_base + (uint32_t)((i - g_begin[g]) * N_PAD);
+          const uint32_t dcol = tmem_base + (uint32_t)((i - g_begin[g]) * fp.tile_stride);
 #pragma unroll
           for (int k = 0; k < kBlockK / 16; ++k) {
             umma_bf16(dcol, make_smem_desc(wb + k * 32), make_smem_desc(hb + k * 32), idesc,
@@ -442,18 +443,22 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   } else if (warp < 4) {
     // ------------------------------------------------------------------ epilogue warps
     const uint32_t tmem_lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const int ts = fp.tile_stride;
     bool ok = true;
 
     // (a) overflow tiles: TMEM -> smem as soon as their accumulation is complete
     if (n_ovf > 0) {
-      ok = mbar_wait(smem_u32(&ms.acc_full[0]), 0u, abort_flag);
+      // one thread polls the barrier; the other 127 sleep in the hardware barrier below
+      if (tid == 0) mbar_wait(smem_u32(&ms.acc_full[0]), 0u, abort_flag);
+      epi_sync();
+      ok = (*abort_flag == 0);
       if (ok) {
         tc_fence_after();
         for (int i = 0; i < n_ovf; ++i) {
 #pragma unroll
           for (int c0 = 0; c0 < N_PAD; c0 += 16) {
             float v[16];
-            tmem_ld16(tmem_lane_base + (uint32_t)(i * N_PAD + c0), v);
+            tmem_ld16(tmem_lane_base + (uint32_t)(i * ts + c0), v);
 #pragma unroll
             for (int k = 0; k < 16; ++k) ovf_w[((size_t)i * N_PAD + c0 + k) * kVocabTile + tid] = v[k];
           }
@@ -533,9 +538,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
 
     // (c) wait for the logits of the resident tiles
-    if (ok && T > n_ovf) ok = mbar_wait(smem_u32(&ms.acc_full[1]), 0u, abort_flag);
-    tc_fence_after();
+    if (tid == 0 && ok && T > n_ovf) mbar_wait(smem_u32(&ms.acc_full[1]), 0u, abort_flag);
     epi_sync();
+    tc_fence_after();
     ok = ok && (*abort_flag == 0);
 
     // (d) gather of the drafted tokens' logits (rows listed in the prologue), per-row max
@@ -545,7 +550,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int r = ms.glist[e], x = ms.x_row[r];
         const int i = x / kVocabTile - t0;
         float one[8];
-        load_cols8<N_PAD>(i, i + 1, r, n_ovf, tmem_lane_base, ovf, tid, one);
+        load_cols8<N_PAD>(i, i + 1, r, n_ovf, ts, tmem_lane_base, ovf, tid, one);
         if (tid == (x % kVocabTile)) ws.gath[r] = one[0];
       }
     }
@@ -557,7 +562,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (ok) {
         for (int i0 = 0; i0 < T; i0 += 2) {
           float v0[16], v1[16];
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, tmem_lane_base, ovf, tid, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, v0, v1);
           const bool val0 = (t0 + i0) * kVocabTile + tid < V;
           const bool val1 = (i0 + 1 < T) && ((t0 + i0 + 1) * kVocabTile + tid < V);
           if (val0) {
@@ -586,7 +591,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (ok) {
         for (int i0 = 0; i0 < T; i0 += 2) {
           float v0[16], v1[16];
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, tmem_lane_base, ovf, tid, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, v0, v1);
           const bool val0 = (t0 + i0) * kVocabTile + tid < V;
           const bool val1 = (i0 + 1 < T) && ((t0 + i0 + 1) * kVocabTile + tid < V);
           if (val0) {
@@ -703,7 +708,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
             dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
           }
-          load_cols8<N_PAD>(i0, T, row, n_ovf, tmem_lane_base, ovf, tid, lg);
+          load_cols8<N_PAD>(i0, T, row, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
@@ -828,7 +833,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
             dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
           }
-          load_cols8<N_PAD>(i0, T, row, n_ovf, tmem_lane_base, ovf, tid, lg);
+          load_cols8<N_PAD>(i0, T, row, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
@@ -924,7 +929,12 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
   const int n_pad = (R + 15) / 16 * 16;
   const int num_tiles = (V + kVocabTile - 1) / kVocabTile;
   const int max_tiles = (num_tiles + num_sms - 1) / num_sms;
-  const int tmem_tiles = std::min(max_tiles, kTmemCols / n_pad);
+  // Tiles sit `stride` TMEM columns apart, stride = rows rounded up to 8. When stride < n_pad the
+  // last n_pad - stride columns an MMA writes fall on the next tile's first columns; they belong
+  // to zero-padded rows of H, so after that tile's own first (overwriting) MMA, which is issued
+  // later in the same k-step, every further write there adds exactly zero.
+  const int stride = (R + 7) / 8 * 8;
+  const int tmem_tiles = std::min(max_tiles, (kTmemCols - n_pad) / stride + 1);
   const int n_ovf = max_tiles - tmem_tiles;
   if (n_ovf > tmem_tiles) return false;   // the overflow group itself must fit in TMEM
   const size_t fixed = 1024 /*alignment slack*/ + kMiscBytes + (size_t)kHStages * n_pad * 128 +
@@ -938,6 +948,7 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
     plan->n_pad = n_pad;
     plan->max_tiles = max_tiles;
     plan->tmem_tiles = tmem_tiles;
+    plan->tile_stride = stride;
     plan->stages = stages;
     plan->smem_bytes = fixed + (size_t)stages * kWStageBytes;
   }
@@ -951,6 +962,7 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
   fp.num_tiles = (cp.V + kVocabTile - 1) / kVocabTile;
   fp.stages = plan.stages;
   fp.tmem_tiles = plan.tmem_tiles;
+  fp.tile_stride = plan.tile_stride;
   fp.R = cp.B * (cp.M + 1);
   fp.off_h = kMiscBytes;
   fp.off_ovf = fp.off_h + kHStages * plan.n_pad * 128;

@@ -23,6 +23,7 @@ struct FusedPlan {
   int n_pad;          // MMA N: rows padded to a multiple of 16
   int max_tiles;      // vocabulary tiles of the busiest CTA
   int tmem_tiles;     // tiles whose accumulators stay in tensor memory
+  int tile_stride;    // TMEM columns between consecutive tiles
   size_t smem_bytes;  // dynamic shared memory of the launch
   int stages;         // W ring depth
 };

@@ -12,8 +12,8 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libjd_b200.so")
-SOURCES = ["jd_api.cu", "jd_simt.cu", "jd_fused_sm100.cu", "jd_static.cu"]
-HEADERS = ["jd_common.cuh", "jd_kernels.h"]
+SOURCES = ["jd_api.cu", "jd_simt.cu", "jd_fused_sm100.cu", "jd_batched_sm100.cu", "jd_static.cu"]
+HEADERS = ["jd_common.cuh", "jd_kernels.h", "jd_sm100_ptx.cuh"]
 
 
 def _nvcc() -> str:

@@ -23,6 +23,7 @@ struct jd_handle_s {
   bool head_set;
   bool tm_w_ok;
   CUtensorMap tm_w;        // W as a [V, d] bf16 tensor, box 64 x 128, 128-byte swizzle
+  CUtensorMap tm_w256;     // same tensor, box 64 x 256 (batched variant)
   cudaStream_t last_stream;
   int last_variant;
   int last_launches;
@@ -109,6 +110,7 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
   w.mass_p = (double*)take(maxB * np * 8);
   w.w_sel = (float*)take(maxB * (size_t)c.V * 4);
   w.p_sel = (float*)take(maxB * (size_t)c.V * 4);
+  w.h_sel = (__nv_bfloat16*)take(maxB * (size_t)c.d * 2);
   w.status = (unsigned*)take(256);
   w.barrier = (unsigned*)take(256);
   w.np_cap = (int)np;
@@ -210,7 +212,8 @@ jd_status_t jd_set_head(jd_handle_t h, const void* W, const void* w_judge, float
   h->head_set = true;
   h->tm_w_ok = false;
   if (h->cfg.dtype == JD_DTYPE_BF16 && h->cfg.d % 64 == 0)
-    h->tm_w_ok = make_tensor_map(&h->tm_w, W, (uint64_t)h->cfg.V, (uint64_t)h->cfg.d, 128);
+    h->tm_w_ok = make_tensor_map(&h->tm_w, W, (uint64_t)h->cfg.V, (uint64_t)h->cfg.d, 128) &&
+                 make_tensor_map(&h->tm_w256, W, (uint64_t)h->cfg.V, (uint64_t)h->cfg.d, 256);
   return JD_OK;
 }
 
@@ -235,10 +238,16 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
 
   FusedPlan plan;
   const bool fused_ok = h->tm_w_ok && fused_supported(c.dtype, R, c.d, c.V, h->num_sms, &plan);
+  const bool batched_ok = h->tm_w_ok && batched_supported(c.dtype, a->B, c.d, c.V, h->num_sms);
   int variant = a->variant;
-  if (variant == JD_VARIANT_AUTO) variant = (fused_ok && !a->logits_debug) ? JD_VARIANT_FUSED : JD_VARIANT_SIMT;
+  if (variant == JD_VARIANT_AUTO) {
+    if (a->logits_debug) variant = JD_VARIANT_SIMT;
+    else if (fused_ok) variant = JD_VARIANT_FUSED;
+    else if (batched_ok) variant = JD_VARIANT_BATCHED;
+    else variant = JD_VARIANT_SIMT;
+  }
   if (variant == JD_VARIANT_FUSED && (!fused_ok || a->logits_debug)) return JD_ERR_UNSUPPORTED;
-  if (variant == JD_VARIANT_BATCHED) return JD_ERR_UNSUPPORTED;
+  if (variant == JD_VARIANT_BATCHED && (!batched_ok || a->logits_debug)) return JD_ERR_UNSUPPORTED;
 
   if (cudaSetDevice(c.device) != cudaSuccess) return JD_ERR_CUDA;
   // status word and the grid-barrier counters behind it start every call at zero
@@ -246,6 +255,16 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   int launches = 0;
   if (variant == JD_VARIANT_SIMT) {
     launches = run_simt(cp, h->ws, h->W, h->w_judge, a->H, c.dtype, a->logits_debug, st);
+  } else if (variant == JD_VARIANT_BATCHED) {
+    FusedPlan plan2;   // second pass: B rows through the fused kernel
+    if (!fused_supported(c.dtype, a->B, c.d, c.V, h->num_sms, &plan2)) return JD_ERR_UNSUPPORTED;
+    CUtensorMap tm_h, tm_hsel;
+    if (!make_tensor_map(&tm_h, a->H, (uint64_t)R, (uint64_t)c.d, 128) ||
+        !make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)a->B, (uint64_t)c.d, (uint32_t)plan2.n_pad))
+      return JD_ERR_CUDA;
+    cudaError_t err = cudaSuccess;
+    launches = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, a->H, h->w_judge, h->num_sms, st, &err);
+    if (launches < 0) return JD_ERR_CUDA;
   } else {
     CUtensorMap tm_h;
     if (!make_tensor_map(&tm_h, a->H, (uint64_t)R, (uint64_t)c.d, (uint32_t)plan.n_pad)) return JD_ERR_CUDA;

@@ -1,0 +1,246 @@
+// Batched variant for many rows (B*(M+1) in the hundreds or thousands): the R x V logits are far
+// too many to keep on chip, so the call runs in two tensor-core passes.
+//
+// Pass 1, gemm_stats_kernel: persistent tcgen05 GEMM, rows of H on the MMA's M axis (128 TMEM
+//   lanes = 128 rows), 256 vocabulary entries on N. Each 128 x 256 logits tile lives only in
+//   tensor memory: the epilogue warps turn it into one (max, sum exp) pair per row and pick out
+//   the drafted token's logit, while the next tile's MMAs fill the other half of tensor memory.
+// Then the shared decision kernel folds the per-tile pairs, runs both tests and the prefix rule.
+// Pass 2: the selected row of every sequence (B rows) is gathered and handed to the fused
+//   kernel in its sample-only mode, which recomputes those B rows of logits with W streamed
+//   once more and draws the next tokens.
+// The logits never reach device memory in either pass.
+#include "jd_kernels.h"
+#include "jd_sm100_ptx.cuh"
+
+namespace jd {
+
+namespace {
+
+constexpr int kBThreads = 192;
+constexpr int kTileM = 128;   // rows per tile
+constexpr int kTileN = 256;   // vocabulary entries per tile
+constexpr int kTileK = 64;    // bf16 per k-step (one 128-byte swizzle row)
+constexpr int kAStage = kTileM * 128;   // 16 KB
+constexpr int kBStage = kTileN * 128;   // 32 KB
+constexpr int kBStages = 4;
+constexpr int kBMisc = 1024;
+
+struct BMisc {
+  uint64_t full[kBStages], empty[kBStages];
+  uint64_t tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__global__ void __launch_bounds__(kBThreads, 1)
+gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, CallParams cp,
+                  Workspace ws, int R, int np) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  BMisc& ms = *reinterpret_cast<BMisc*>(smem);
+  const uint32_t sA = smem_u32(smem + kBMisc);
+  const uint32_t sB = sA + kBStages * kAStage;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = gridDim.x;
+  volatile int* abort_flag = &ms.abort_flag;
+  const int num_kb = cp.d / kTileK;
+  const int row_blocks = (R + kTileM - 1) / kTileM;
+  const int voc_blocks = (cp.V + kTileN - 1) / kTileN;
+  const int num_tiles = row_blocks * voc_blocks;
+
+  if (tid == 0) {
+    for (int s = 0; s < kBStages; ++s) { mbar_init(smem_u32(&ms.full[s]), 1); mbar_init(smem_u32(&ms.empty[s]), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ms.tmem_full[s]), 1); mbar_init(smem_u32(&ms.tmem_empty[s]), 1); }
+    ms.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ms.tmem_base)),
+                 "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = ms.tmem_base;
+
+  // Tile order: consecutive tile ids share the vocabulary block, so the CTAs that run at the
+  // same time read the same W slab and all but the first find it in L2.
+  if (warp == 4 && lane == 0) {
+    const uint64_t pol_w = policy_evict_first(), pol_h = policy_evict_last();
+    int s = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < num_tiles && ok; t += G) {
+      const int vb = t / row_blocks, rb = t % row_blocks;
+      for (int kb = 0; kb < num_kb; ++kb) {
+        ok = mbar_wait(smem_u32(&ms.empty[s]), ph ^ 1u, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(smem_u32(&ms.full[s]), kAStage + kBStage);
+        tma_load_2d(sA + s * kAStage, &tmH, smem_u32(&ms.full[s]), kb * kTileK, rb * kTileM, pol_h);
+        tma_load_2d(sB + s * kBStage, &tmW, smem_u32(&ms.full[s]), kb * kTileK, vb * kTileN, pol_w);
+        if (++s == kBStages) { s = 0; ph ^= 1u; }
+      }
+    }
+    if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
+  } else if (warp == 5 && lane == 0) {
+    const uint32_t idesc = make_idesc(kTileN);
+    int s = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    int it = 0;
+    for (int t = blockIdx.x; t < num_tiles && ok; t += G, ++it) {
+      const int buf = it & 1;
+      ok = mbar_wait(smem_u32(&ms.tmem_empty[buf]), ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t dcol = tmem_base + (uint32_t)(buf * kTileN);
+      for (int kb = 0; kb < num_kb; ++kb) {
+        ok = mbar_wait(smem_u32(&ms.full[s]), ph, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t ab = sA + s * kAStage, bb = sB + s * kBStage;
+#pragma unroll
+        for (int k = 0; k < kTileK / 16; ++k)
+          umma_bf16(dcol, make_smem_desc(ab + k * 32), make_smem_desc(bb + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+        umma_commit(smem_u32(&ms.empty[s]));
+        if (++s == kBStages) { s = 0; ph ^= 1u; }
+      }
+      if (ok) umma_commit(smem_u32(&ms.tmem_full[buf]));
+    }
+    if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
+  } else if (warp < 4) {
+    // Epilogue: thread = row. Online (max, sum exp) over the tile's 256 columns, 32 at a time.
+    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    bool ok = true;
+    int it = 0;
+    for (int t = blockIdx.x; t < num_tiles; t += G, ++it) {
+      const int vb = t / row_blocks, rb = t % row_blocks;
+      const int buf = it & 1;
+      const int row = rb * kTileM + tid;
+      const int v0 = vb * kTileN;
+      int x = -1;
+      if (row < R) {
+        const int b = row / (cp.M + 1), j = row % (cp.M + 1);
+        if (j < cp.M) {
+          x = cp.draft_tokens[b * cp.M + j];
+          if (x < 0 || x >= cp.V) { set_status(ws.status, JD_ERR_BAD_TOKEN); x = min(max(x, 0), cp.V - 1); }
+        }
+      }
+      if (tid == 0) mbar_wait(smem_u32(&ms.tmem_full[buf]), (uint32_t)(it >> 1) & 1u, abort_flag);
+      epi_sync();
+      ok = (*abort_flag == 0);
+      if (!ok) break;
+      tc_fence_after();
+      float m = -INFINITY, s = 0.f, g = 0.f;
+      bool have_g = false;
+#pragma unroll 1
+      for (int c0 = 0; c0 < kTileN; c0 += 32) {
+        float v[32];
+        tmem_ld32(lane_base + (uint32_t)(buf * kTileN + c0), v);
+        const int nvalid = cp.V - (v0 + c0);   // columns of this chunk that exist (>= 32 except at the tail)
+        if (nvalid < 32) {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) if (k >= nvalid) v[k] = -INFINITY;
+        }
+        float cm = v[0];
+#pragma unroll
+        for (int k = 1; k < 32; ++k) cm = fmaxf(cm, v[k]);
+        const float mn = fmaxf(m, cm);
+        if (mn > -INFINITY) {
+          const float off = mn * kLog2e;
+          float acc = 0.f;
+#pragma unroll
+          for (int k = 0; k < 32; ++k) acc += fast_exp2(fmaf(v[k], kLog2e, -off));
+          s = s * fast_exp2(fmaf(m, kLog2e, -off)) + acc;
+          m = mn;
+        }
+        if ((unsigned)(x - (v0 + c0)) < 32u) {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) if (x == v0 + c0 + k) g = v[k];
+          have_g = true;
+        }
+      }
+      tc_fence_before();
+      epi_sync();
+      if (tid == 0) mbar_arrive(smem_u32(&ms.tmem_empty[buf]));
+      if (row < R) {
+        ws.part_max[(size_t)row * np + vb] = m;
+        ws.part_sum[(size_t)row * np + vb] = s;
+        if (have_g) ws.gath[row] = g;
+      }
+    }
+    if (!ok && tid == 0) set_status(ws.status, JD_ERR_TIMEOUT);
+  }
+
+  __syncthreads();
+  if (ms.abort_flag) {
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);
+    __syncthreads();
+  }
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// Copies the selected row of every sequence into a dense [B, d] matrix for the second pass.
+__global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ H, const int* __restrict__ sel_row,
+                                   __nv_bfloat16* __restrict__ out, int d) {
+  const int b = blockIdx.x;
+  const uint4* src = reinterpret_cast<const uint4*>(H + (size_t)sel_row[b] * d);
+  uint4* dst = reinterpret_cast<uint4*>(out + (size_t)b * d);
+  for (int k = threadIdx.x; k < d / 8; k += blockDim.x) dst[k] = src[k];
+}
+
+}  // namespace
+
+bool batched_supported(int dtype, int B, int d, int V, int num_sms) {
+  if (dtype != JD_DTYPE_BF16 || d % kTileK != 0 || d < kTileK) return false;
+  if (num_sms < 1 || num_sms > kMaxCtas) return false;
+  FusedPlan plan;
+  return fused_supported(dtype, B, d, V, num_sms, &plan);   // the second pass runs B rows through the fused kernel
+}
+
+int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
+                const CUtensorMap& tmH, const CUtensorMap& tmHsel, const void* H, const void* w_judge, int num_sms,
+                cudaStream_t st, cudaError_t* err) {
+  const int R = cp.B * (cp.M + 1);
+  const int np = (cp.V + kTileN - 1) / kTileN;
+  const int nq = launch_q_stats(cp, ws, st);
+  launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, st);
+  const size_t smem = 1024 + kBMisc + (size_t)kBStages * (kAStage + kBStage);
+  *err = cudaFuncSetAttribute(gemm_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (*err != cudaSuccess) return -1;
+  const int row_blocks = (R + kTileM - 1) / kTileM, voc_blocks = np;
+  const int grid = std::min(num_sms, row_blocks * voc_blocks);
+  gemm_stats_kernel<<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+  launch_decide(cp, ws, np, nq, st);
+  gather_rows_kernel<<<cp.B, 256, 0, st>>>((const __nv_bfloat16*)H, ws.sel_row, ws.h_sel, cp.d);
+  FusedPlan plan;
+  if (!fused_supported(JD_DTYPE_BF16, cp.B, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }
+  const int n = run_fused(cp, ws, tmW128, tmHsel, ws.h_sel, w_judge, plan, st, err, /*sample_only=*/true);
+  if (n < 0) return -1;
+  return 5 + n;
+}
+
+}  // namespace jd

@@ -37,6 +37,7 @@ struct Workspace {
   double* mass_p;      // [maxB][np] mass of p per slice (zero-residual fallback)
   float* w_sel;        // [maxB][V]  sampling weights (SIMT / batched second pass only)
   float* p_sel;        // [maxB][V]  p of the selected row (same)
+  __nv_bfloat16* h_sel;  // [maxB][d] selected rows of H gathered for the batched variant's second pass
   unsigned* status;    // [1] device status word (jd_status_t of the first device-side problem)
   unsigned* barrier;   // [8] grid-barrier counters of the fused variant
   int np_cap;          // capacity (partials per row) of part_* and mass_*

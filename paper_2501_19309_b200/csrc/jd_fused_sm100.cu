@@ -26,6 +26,7 @@
 #include <cooperative_groups.h>
 
 #include "jd_kernels.h"
+#include "jd_sm100_ptx.cuh"
 
 namespace jd {
 
@@ -36,10 +37,10 @@ constexpr int kEpiThreads = 128;
 constexpr int kBlockK = 64;                      // bf16 elements per k-slice = one 128-byte swizzle row
 constexpr int kWStageBytes = kVocabTile * 128;   // 16 KB
 constexpr int kTmemCols = 512;
-constexpr int kMiscBytes = 13312;                // barriers + reduction scratch at the head of smem
+constexpr int kMiscBytes = 16384;                // barriers + reduction scratch at the head of smem
 constexpr int kMaxStages = 12;
 constexpr int kHStages = 4;
-constexpr float kLog2e = 1.4426950408889634f;
+
 
 struct FusedParams {
   int num_kb;       // d / 64
@@ -47,129 +48,12 @@ struct FusedParams {
   int stages;       // W ring depth
   int tmem_tiles;   // tiles resident in TMEM
   int tile_stride;  // TMEM columns between consecutive tiles (>= rows, multiple of 8, <= N_PAD)
-  int R;            // B * (M + 1)
+  int R;            // rows of the H matrix given to the MMA: B * (M + 1), or B in sample-only mode
+  int sample_only;  // 1: H holds one already selected row per sequence; only the token draw runs
   uint32_t off_h;   // byte offsets inside dynamic smem (from the 1024-aligned base)
   uint32_t off_ovf;
   uint32_t off_w;
 };
-
-// ------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: false when the limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (unsigned it = 0; it < kSpinLimit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (it > 128) {
-      __nanosleep(64);
-      if (*abort_flag) return false;
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
-
-__device__ __forceinline__ uint64_t policy_evict_first() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ uint64_t policy_evict_last() {
-  uint64_t p;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-  return p;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
-                                            uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-      " [%0], [%1, {%3, %4}], [%2], %5;"
-      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// K-major, 128-byte swizzle shared-memory matrix descriptor: start address, stride between
-// 8-row groups = 1024 bytes, descriptor version 1, layout type 2 (SWIZZLE_128B).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)(1024u >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
-  return d;
-}
-// Instruction descriptor, kind::f16: D = f32, A = B = bf16, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t make_idesc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-  uint32_t r[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-#pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-// issue only; the value is valid after tmem_wait_ld8 has been given the registers
-__device__ __forceinline__ void tmem_ld1_issue(uint32_t taddr, uint32_t& r) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld8(uint32_t* r) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
-               :: "memory");
-}
-__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-// Grid barrier on a global counter; thread 0 of the epilogue group calls it. Cooperative launch
-// guarantees co-residency; the spin is bounded all the same.
-__device__ __forceinline__ bool grid_arrive_and_wait(unsigned* counter, unsigned expected, volatile int* abort_flag) {
-  __threadfence();
-  atomicAdd(counter, 1u);
-  for (unsigned it = 0; it < kSpinLimit; ++it) {
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
-    if (v >= expected) return true;
-    __nanosleep(40);
-    if (*abort_flag) return false;
-  }
-  *abort_flag = 1;
-  return false;
-}
 
 // ------------------------------------------------------------------------------ shared scratch
 template <int N_PAD>
@@ -188,48 +72,23 @@ struct Misc {
   float qlse[N_PAD];
   int x_row[N_PAD];         // drafted token of row r (rows j < M), -1 otherwise
   int glist[N_PAD];
-  // per sequence (B <= N_PAD / 2 because M >= 1)
-  int sel_row[N_PAD / 2];
-  int sel_kind[N_PAD / 2];
-  float sel_lse_p[N_PAD / 2];
-  float sel_lse_q[N_PAD / 2];
-  float sel_u[N_PAD / 2];
-  double wd_r[N_PAD / 2][4];
-  double wd_p[N_PAD / 2][4];
-  int own_cta[N_PAD / 2];
-  int own_usep[N_PAD / 2];
-  double own_prefix[N_PAD / 2];
-  double own_T[N_PAD / 2];
+  // per sequence (B <= N_PAD / 2 in the full mode, B <= N_PAD in sample-only mode)
+  int sel_row[N_PAD];
+  int sel_kind[N_PAD];
+  float sel_lse_p[N_PAD];
+  float sel_lse_q[N_PAD];
+  float sel_u[N_PAD];
+  double wd_r[N_PAD][4];
+  double wd_p[N_PAD][4];
+  int own_cta[N_PAD];
+  int own_usep[N_PAD];
+  double own_prefix[N_PAD];
+  double own_T[N_PAD];
   double tsum[4][8];
   double wscan[4];
   int cand[4];
   int lastpos[4];
 };
-
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-// one wait for two 16-column loads; the registers pass through the statement so that nothing
-// that consumes them can be scheduled ahead of the wait
-__device__ __forceinline__ void tmem_wait_ld32(uint32_t* a, uint32_t* b) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
-                 "+r"(a[8]), "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]),
-                 "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
-                 "+r"(b[8]), "+r"(b[9]), "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15])
-               :: "memory");
-}
 
 // logits of rows c0..c0+15 for this thread's lane in tiles i0 and i0+1 (zeros past T): from TMEM,
 // or from the overflow copy in shared memory
@@ -350,7 +209,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   }
   if (tid < N_PAD) {
     int x = -1;
-    if (tid < R) {
+    if (tid < R && !fp.sample_only) {
       const int b = tid / (M + 1), j = tid % (M + 1);
       if (j < M) {
         x = cp.draft_tokens[b * M + j];
@@ -472,7 +331,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     // (b) while W streams: draft-row statistics over this CTA's vocabulary slice, judge dots
     const int v_lo = t0 * kVocabTile, v_hi = min(V, (t0 + T) * kVocabTile);
     const bool vec4 = (V % 4) == 0;   // rows are 16-byte aligned only then
-    for (int bm = warp; bm < BM; bm += 4) {
+    for (int bm = warp; bm < (fp.sample_only ? 0 : BM); bm += 4) {
       const float* row = cp.draft_logits + (size_t)bm * V;
       float m = -INFINITY, s = 0.f;
       if (vec4) {
@@ -516,7 +375,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         if (x >= v_lo && x < v_hi) ws.qgath[bm] = row[x];
       }
     }
-    for (int bm = cta * 4 + warp; bm < BM; bm += G * 4) {
+    for (int bm = cta * 4 + warp; bm < (fp.sample_only ? 0 : BM); bm += G * 4) {
       const int b = bm / M, j = bm % M;
       const uint4* h4 = reinterpret_cast<const uint4*>(H + ((size_t)b * (M + 1) + j + 1) * cp.d);
       const uint4* w4 = reinterpret_cast<const uint4*>(wj);
@@ -543,6 +402,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     tc_fence_after();
     ok = ok && (*abort_flag == 0);
 
+    if (!fp.sample_only) {
     // (d) gather of the drafted tokens' logits (rows listed in the prologue), per-row max
     if (ok) {
       const int ng = ms.glist_n;
@@ -694,10 +554,23 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     epi_sync();
 
+    } else {
+      // sample-only mode: an earlier kernel made the decisions; fetch what the token draw needs
+      if (ok && tid < cp.B) {
+        ms.sel_row[tid] = ws.sel_row[tid];
+        ms.sel_kind[tid] = ws.sel_kind[tid];
+        ms.sel_lse_p[tid] = ws.sel_lse_p[tid];
+        ms.sel_lse_q[tid] = ws.sel_lse_q[tid];
+        ms.sel_u[tid] = ws.sel_u[tid];
+      }
+      epi_sync();
+    }
+
     // (h) mass of the sampling weights of each selected row over this CTA's slice
     if (ok) {
       for (int b = 0; b < cp.B; ++b) {
         const int row = ms.sel_row[b], kind = ms.sel_kind[b];
+        const int col = fp.sample_only ? b : row;   // TMEM column that holds this sequence's selected row
         const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
         const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;   // used only when kind == 0
         double sr = 0.0, sp = 0.0;
@@ -708,7 +581,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
             dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
           }
-          load_cols8<N_PAD>(i0, T, row, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
+          load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
@@ -819,6 +692,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       for (int b = 0; b < cp.B; ++b) {
         if (ms.own_cta[b] != cta) continue;
         const int row = ms.sel_row[b];
+        const int col = fp.sample_only ? b : row;
         const int kind = ms.own_usep[b] ? 1 : ms.sel_kind[b];
         const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
         const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;
@@ -833,7 +707,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
             dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
           }
-          load_cols8<N_PAD>(i0, T, row, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
+          load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
@@ -956,14 +830,16 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
 }
 
 int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
-              const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err) {
+              const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err,
+              bool sample_only) {
   FusedParams fp;
   fp.num_kb = cp.d / kBlockK;
   fp.num_tiles = (cp.V + kVocabTile - 1) / kVocabTile;
   fp.stages = plan.stages;
   fp.tmem_tiles = plan.tmem_tiles;
   fp.tile_stride = plan.tile_stride;
-  fp.R = cp.B * (cp.M + 1);
+  fp.R = sample_only ? cp.B : cp.B * (cp.M + 1);
+  fp.sample_only = sample_only ? 1 : 0;
   fp.off_h = kMiscBytes;
   fp.off_ovf = fp.off_h + kHStages * plan.n_pad * 128;
   const int n_ovf = plan.max_tiles - plan.tmem_tiles;

@@ -30,6 +30,15 @@ struct FusedPlan {
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan);
 // Returns the number of kernels launched, or -1 with *err set.
 int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
-              const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err);
+              const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err,
+              bool sample_only = false);
+
+// Two-pass tensor-core variant for many rows (jd_batched_sm100.cu). tmW256 / tmW128: W with
+// 256- and 128-row boxes; tmH: H with a 128-row box; tmHsel: the handle's [B, d] gather buffer
+// with the fused plan's box. Returns the number of kernels launched, or -1 with *err set.
+bool batched_supported(int dtype, int B, int d, int V, int num_sms);
+int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
+                const CUtensorMap& tmH, const CUtensorMap& tmHsel, const void* H, const void* w_judge, int num_sms,
+                cudaStream_t st, cudaError_t* err);
 
 }  // namespace jd

@@ -83,5 +83,5 @@ def test_cfg3_masks_independent_of_mode():
 
 
 def test_cfg4_batched_sampled_sequences():
-    rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[0, 37, 63])
+    rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[0, 37, 63], expect_variant="batched")
     assert rep.sequences == 3

@@ -239,3 +239,38 @@ def test_fused_unsupported_shapes_are_refused_not_faked():
     a, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, variant="fused")
     assert jd.jd_verify(ver.h, a) == jd.JD_ERR_UNSUPPORTED
     ver.close()
+
+
+# ------------------------------------------------------------------ batched tensor-core variant
+BATCHED_SHAPES = [
+    (8, 16, 128, 128256),       # 136 rows: two row blocks, the second mostly padding
+    (3, 50, 128, 5000 + 77),    # 153 rows, ragged last vocabulary block
+    (64, 16, 64, 128256),       # the serving shape's rows (1088) at a narrow d
+    (2, 3, 64, 700),            # fewer tiles than CTAs
+    (40, 2, 128, 33000),        # many short sequences
+]
+
+
+@pytest.mark.parametrize("B,M,d,V", BATCHED_SHAPES)
+def test_batched_variant_parity(B, M, d, V):
+    wl = I.CONFIGS[4].scaled("batched-%d-%d-%d-%d" % (B, M, d, V), B=B, M=M, d=d, V=V)
+    seqs = None if B <= 8 else sorted({0, 1, B // 2, B - 1})
+    rep = run_case(wl, 5, variant="batched", modes=("judge_or_standard", "standard"), seeds=[0, 1],
+                   sequences=seqs, expect_variant="batched")
+    assert rep.sequences == 4 * (B if seqs is None else len(seqs))
+
+
+def test_batched_matches_simt_on_every_sequence():
+    wl = I.CONFIGS[4].scaled("x", B=48, M=7, d=128, V=20000)
+    inp = I.make_inputs(wl, 2)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    for seed in range(2):
+        a = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, seed, "judge_or_standard", variant="batched"))
+        b = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, seed, "judge_or_standard", variant="simt"))
+        assert np.array_equal(a["accept_len"], b["accept_len"])
+        assert np.array_equal(a["masks"], b["masks"])
+        assert np.mean(a["next_token"] == b["next_token"]) > 0.9      # CDF-edge cases may differ by a token
+        assert np.allclose(a["row_lse"], b["row_lse"], rtol=0, atol=1e-4)
+        assert np.allclose(a["p_draft"], b["p_draft"], rtol=1e-4)
+    ver.close()

@@ -240,7 +240,7 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
   if (!fused_supported(JD_DTYPE_BF16, cp.B, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }
   const int n = run_fused(cp, ws, tmW128, tmHsel, ws.h_sel, w_judge, plan, st, err, /*sample_only=*/true);
   if (n < 0) return -1;
-  return 5 + n;
+  return 6 + n;
 }
 
 }  // namespace jd

@@ -566,36 +566,52 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       epi_sync();
     }
 
-    // (h) mass of the sampling weights of each selected row over this CTA's slice
+    // (h) mass of the sampling weights of each selected row over this CTA's slice; four
+    // sequences at a time so that their draft-logit loads are in flight together
     if (ok) {
-      for (int b = 0; b < cp.B; ++b) {
-        const int row = ms.sel_row[b], kind = ms.sel_kind[b];
-        const int col = fp.sample_only ? b : row;   // TMEM column that holds this sequence's selected row
-        const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
-        const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;   // used only when kind == 0
-        double sr = 0.0, sp = 0.0;
+      for (int b0 = 0; b0 < cp.B; b0 += 4) {
+        double sr[4] = {0.0, 0.0, 0.0, 0.0}, sp[4] = {0.0, 0.0, 0.0, 0.0};
         for (int i0 = 0; i0 < T; i0 += 8) {
-          float dv[8], lg[8];
+          float dv[4][8], lg[4][8];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int vg = (t0 + i0 + u) * kVocabTile + tid;
-            dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
+          for (int q = 0; q < 4; ++q) {
+            const int b = min(b0 + q, cp.B - 1);
+            const int row = ms.sel_row[b], kind = ms.sel_kind[b];
+            const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;   // read only when kind == 0
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int vg = (t0 + i0 + u) * kVocabTile + tid;
+              dv[q][u] = (kind == 0 && b0 + q < cp.B && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
+            }
           }
-          load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int vg = (t0 + i0 + u) * kVocabTile + tid;
-            if (i0 + u < T && vg < V) {
-              float p, r;
-              sample_weights(lg[u], lse_p, kind, dv[u], lse_q, p, r);
-              sr += (double)r;
-              sp += (double)p;
+          for (int q = 0; q < 4; ++q) {
+            const int b = min(b0 + q, cp.B - 1);
+            const int col = fp.sample_only ? b : ms.sel_row[b];   // TMEM column of this sequence's selected row
+            load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, lg[q]);
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int b = min(b0 + q, cp.B - 1);
+            const int kind = ms.sel_kind[b];
+            const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int vg = (t0 + i0 + u) * kVocabTile + tid;
+              if (i0 + u < T && vg < V) {
+                float p, r;
+                sample_weights(lg[q][u], lse_p, kind, dv[q][u], lse_q, p, r);
+                sr[q] += (double)r;
+                sp[q] += (double)p;
+              }
             }
           }
         }
-        sr = warp_sum_double(sr);
-        sp = warp_sum_double(sp);
-        if (lane == 0) { ms.wd_r[b][warp] = sr; ms.wd_p[b][warp] = sp; }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const double a_r = warp_sum_double(sr[q]), a_p = warp_sum_double(sp[q]);
+          if (lane == 0 && b0 + q < cp.B) { ms.wd_r[b0 + q][warp] = a_r; ms.wd_p[b0 + q][warp] = a_p; }
+        }
       }
     }
     epi_sync();

@@ -135,10 +135,29 @@ __global__ void __launch_bounds__(256) q_stats_kernel(CallParams cp, Workspace w
   const float* row = cp.draft_logits + (size_t)bm * V;
   const int lo = chunk * kQChunk, hi = min(V, lo + kQChunk);
   float m = -INFINITY, s = 0.f;
-  for (int v = lo + threadIdx.x; v < hi; v += blockDim.x) {
-    const float xv = row[v];
-    if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
-    else if (xv != -INFINITY) s += __expf(xv - m);
+  if ((V & 3) == 0) {
+    // rows are 16-byte aligned: every thread fetches its eight float4 of the chunk before any
+    // arithmetic, then takes the maximum and the sum of exponentials from registers
+    float4 x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int v = lo + (u * 256 + threadIdx.x) * 4;
+      x[u] = v < hi ? __ldg(reinterpret_cast<const float4*>(row + v))
+                    : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) m = fmaxf(m, fmaxf(fmaxf(x[u].x, x[u].y), fmaxf(x[u].z, x[u].w)));
+    if (m > -INFINITY) {
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        s += (__expf(x[u].x - m) + __expf(x[u].y - m)) + (__expf(x[u].z - m) + __expf(x[u].w - m));
+    }
+  } else {
+    for (int v = lo + threadIdx.x; v < hi; v += blockDim.x) {
+      const float xv = row[v];
+      if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
+      else if (xv != -INFINITY) s += __expf(xv - m);
+    }
   }
   ms_warp_reduce(m, s);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -178,37 +197,60 @@ __global__ void __launch_bounds__(256) judge_dot_kernel(CallParams cp, Workspace
 }
 
 // -----------------------------------------------------------------------------------------
-// Decision: one block per sequence. Warps first fold the partial statistics of the rows
-// (fixed order, so results repeat bit for bit), then warp 0 runs the tests.
+// Fold of the partial statistics: one warp per target row and per draft row. Each lane fetches
+// its share of the row's partials (eight at a time, all loads first), the warp takes the
+// maximum, then the rescaled sum; fixed order, so results repeat bit for bit.
 // -----------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) decide_kernel(CallParams cp, Workspace ws, int np, int nq) {
-  const int b = blockIdx.x;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int M = cp.M;
-  for (int j = warp; j <= M; j += 4) {
-    const int row = b * (M + 1) + j;
-    float m = -INFINITY, s = 0.f;
-    for (int i = lane; i < np; i += 32)
-      ms_combine(m, s, ws.part_max[(size_t)row * np + i], ws.part_sum[(size_t)row * np + i]);
-    ms_warp_reduce(m, s);
-    if (lane == 0) {
-      const float lse = m + logf(s);
-      ws.row_max[row] = m;
-      ws.row_lse[row] = lse;
-      if (cp.row_max_out) cp.row_max_out[row] = m;
-      if (cp.row_lse_out) cp.row_lse_out[row] = lse;
+__global__ void __launch_bounds__(256) fold_stats_kernel(CallParams cp, Workspace ws, int np, int nq) {
+  const int lane = threadIdx.x & 31;
+  const int R = cp.B * (cp.M + 1), BM = cp.B * cp.M;
+  const int it = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (it >= R + BM) return;
+  const bool is_p = it < R;
+  const int n = is_p ? np : nq;
+  const float* pm = is_p ? ws.part_max + (size_t)it * np : ws.qpart_max + (size_t)(it - R) * nq;
+  const float* ps = is_p ? ws.part_sum + (size_t)it * np : ws.qpart_sum + (size_t)(it - R) * nq;
+  float m = -INFINITY;
+  for (int i0 = 0; i0 < n; i0 += 256) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { const int i = i0 + u * 32 + lane; v[u] = i < n ? pm[i] : -INFINITY; }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) m = fmaxf(m, v[u]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  float s = 0.f;
+  for (int i0 = 0; i0 < n; i0 += 256) {
+    float vm[8], vs[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * 32 + lane;
+      vm[u] = i < n ? pm[i] : -INFINITY;
+      vs[u] = i < n ? ps[i] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) if (vs[u] > 0.f) s += vs[u] * __expf(vm[u] - m);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if (lane == 0) {
+    const float lse = m + logf(s);
+    if (is_p) {
+      ws.row_max[it] = m;
+      ws.row_lse[it] = lse;
+      if (cp.row_max_out) cp.row_max_out[it] = m;
+      if (cp.row_lse_out) cp.row_lse_out[it] = lse;
+    } else {
+      ws.q_lse[it - R] = lse;
     }
   }
-  for (int j = warp; j < M; j += 4) {
-    const int bm = b * M + j;
-    float m = -INFINITY, s = 0.f;
-    for (int i = lane; i < nq; i += 32)
-      ms_combine(m, s, ws.qpart_max[(size_t)bm * nq + i], ws.qpart_sum[(size_t)bm * nq + i]);
-    ms_warp_reduce(m, s);
-    if (lane == 0) ws.q_lse[bm] = m + logf(s);
-  }
-  __syncthreads();
-  if (warp == 0) decide_sequence(cp, ws, b, true);
+}
+
+// Decision: one warp per sequence runs the tests and the prefix rule on the folded statistics.
+__global__ void __launch_bounds__(128) decide_kernel(CallParams cp, Workspace ws) {
+  const int b = blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (b < cp.B) decide_sequence(cp, ws, b, true);
 }
 
 // -----------------------------------------------------------------------------------------
@@ -280,7 +322,9 @@ void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, cons
 }
 
 void launch_decide(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st) {
-  decide_kernel<<<cp.B, 128, 0, st>>>(cp, ws, np, nq);
+  const int items = cp.B * (2 * cp.M + 1);
+  fold_stats_kernel<<<(items + 7) / 8, 256, 0, st>>>(cp, ws, np, nq);
+  decide_kernel<<<(cp.B + 3) / 4, 128, 0, st>>>(cp, ws);
 }
 
 void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream_t st) {
@@ -309,7 +353,7 @@ int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const voi
   if (dtype == JD_DTYPE_BF16) simt_logits<__nv_bfloat16>(cp, ws, W, H, true, np, nullptr, st);
   else simt_logits<float>(cp, ws, W, H, true, np, nullptr, st);
   launch_locate(cp, ws, np, st);
-  return 6;
+  return 7;
 }
 
 void launch_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot, const int32_t* stream, int n,

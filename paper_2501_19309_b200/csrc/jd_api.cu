@@ -108,7 +108,7 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
   w.sel_u = (float*)take(maxB * 4);
   w.mass_r = (double*)take(maxB * np * 8);
   w.mass_p = (double*)take(maxB * np * 8);
-  w.w_sel = (float*)take(maxB * (size_t)c.V * 4);
+  w.w_sel = (float*)take(maxB * (((size_t)c.V + kVocabTile - 1) / kVocabTile * kVocabTile) * 4);
   w.p_sel = (float*)take(maxB * (size_t)c.V * 4);
   w.h_sel = (__nv_bfloat16*)take(maxB * (size_t)c.d * 2);
   w.status = (unsigned*)take(256);

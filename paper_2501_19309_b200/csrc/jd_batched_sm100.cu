@@ -203,13 +203,22 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   }
 }
 
-// Copies the selected row of every sequence into a dense [B, d] matrix for the second pass.
-__global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ H, const int* __restrict__ sel_row,
-                                   __nv_bfloat16* __restrict__ out, int d) {
-  const int b = blockIdx.x;
-  const uint4* src = reinterpret_cast<const uint4*>(H + (size_t)sel_row[b] * d);
-  uint4* dst = reinterpret_cast<uint4*>(out + (size_t)b * d);
-  for (int k = threadIdx.x; k < d / 8; k += blockDim.x) dst[k] = src[k];
+// Prepares the second pass: copies the selected row of H of every sequence into a dense [B, d]
+// matrix, and the selected draft-logit row (where the residual needs it) into a tile-major
+// buffer [vocab tile][sequence][128], so that a CTA of the second pass finds the draft logits of
+// its vocabulary slice for all sequences in one contiguous block.
+__global__ void __launch_bounds__(256) gather_rows_kernel(CallParams cp, Workspace ws, const __nv_bfloat16* __restrict__ H) {
+  const int b = blockIdx.x, part = blockIdx.y, parts = gridDim.y;
+  const int row = ws.sel_row[b];
+  if (part == 0) {
+    const uint4* src = reinterpret_cast<const uint4*>(H + (size_t)row * cp.d);
+    uint4* dst = reinterpret_cast<uint4*>(ws.h_sel + (size_t)b * cp.d);
+    for (int k = threadIdx.x; k < cp.d / 8; k += blockDim.x) dst[k] = src[k];
+  }
+  if (ws.sel_kind[b] != 0) return;
+  const float* dl = cp.draft_logits + ((size_t)b * cp.M + (row % (cp.M + 1))) * cp.V;
+  for (int v = part * 256 + threadIdx.x; v < cp.V; v += parts * 256)
+    ws.w_sel[((size_t)(v / kVocabTile) * cp.B + b) * kVocabTile + (v % kVocabTile)] = __ldg(dl + v);
 }
 
 }  // namespace
@@ -235,7 +244,7 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
   const int grid = std::min(num_sms, row_blocks * voc_blocks);
   gemm_stats_kernel<<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
   launch_decide(cp, ws, np, nq, st);
-  gather_rows_kernel<<<cp.B, 256, 0, st>>>((const __nv_bfloat16*)H, ws.sel_row, ws.h_sel, cp.d);
+  gather_rows_kernel<<<dim3(cp.B, 8), 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H);
   FusedPlan plan;
   if (!fused_supported(JD_DTYPE_BF16, cp.B, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }
   const int n = run_fused(cp, ws, tmW128, tmHsel, ws.h_sel, w_judge, plan, st, err, /*sample_only=*/true);

@@ -35,7 +35,8 @@ struct Workspace {
   float* sel_u;        // [maxB] uniform of the token draw
   double* mass_r;      // [maxB][np] mass of the sampling weights per vocabulary slice
   double* mass_p;      // [maxB][np] mass of p per slice (zero-residual fallback)
-  float* w_sel;        // [maxB][V]  sampling weights (SIMT / batched second pass only)
+  float* w_sel;        // [maxB][V]  sampling weights (SIMT variant); in the batched variant the selected
+                       //            draft rows, tile-major [ceil(V/128)][B][128]
   float* p_sel;        // [maxB][V]  p of the selected row (same)
   __nv_bfloat16* h_sel;  // [maxB][d] selected rows of H gathered for the batched variant's second pass
   unsigned* status;    // [1] device status word (jd_status_t of the first device-side problem)

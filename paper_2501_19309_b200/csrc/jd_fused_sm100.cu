@@ -138,32 +138,32 @@ __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, int 
 // Reduces 16 per-lane values over the 32 lanes of a warp with 16 shuffles instead of 80: every
 // step halves the number of values a lane keeps. On return lane l holds the reduction of value
 // index reduce16_index(l) (lanes 2j and 2j+1 hold the same one).
-template <bool kMax>
-__device__ __forceinline__ float warp_reduce16(const float* v, int lane) {
-  auto op = [](float x, float y) { return kMax ? fmaxf(x, y) : x + y; };
-  float a[8], b4[4], c2[2];
+template <bool kMax, typename T>
+__device__ __forceinline__ T warp_reduce16(const T* v, int lane) {
+  auto op = [](T x, T y) { return kMax ? (x > y ? x : y) : x + y; };
+  T a[8], b4[4], c2[2];
   const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4, h2 = lane & 2;
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
-    const float send = h16 ? v[k] : v[k + 8];
-    const float keep = h16 ? v[k + 8] : v[k];
+    const T send = h16 ? v[k] : v[k + 8];
+    const T keep = h16 ? v[k + 8] : v[k];
     a[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 16));
   }
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    const float send = h8 ? a[k] : a[k + 4];
-    const float keep = h8 ? a[k + 4] : a[k];
+    const T send = h8 ? a[k] : a[k + 4];
+    const T keep = h8 ? a[k + 4] : a[k];
     b4[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 8));
   }
 #pragma unroll
   for (int k = 0; k < 2; ++k) {
-    const float send = h4 ? b4[k] : b4[k + 2];
-    const float keep = h4 ? b4[k + 2] : b4[k];
+    const T send = h4 ? b4[k] : b4[k + 2];
+    const T keep = h4 ? b4[k + 2] : b4[k];
     c2[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 4));
   }
-  const float send = h2 ? c2[0] : c2[1];
-  const float keep = h2 ? c2[1] : c2[0];
-  float d = op(keep, __shfl_xor_sync(0xffffffffu, send, 2));
+  const T send = h2 ? c2[0] : c2[1];
+  const T keep = h2 ? c2[1] : c2[0];
+  T d = op(keep, __shfl_xor_sync(0xffffffffu, send, 2));
   d = op(d, __shfl_xor_sync(0xffffffffu, d, 1));
   return d;
 }
@@ -435,7 +435,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           }
         }
       }
-      const float red = warp_reduce16<true>(mx, lane);
+      const float red = warp_reduce16<true, float>(mx, lane);
       if ((lane & 1) == 0) ms.wmax[warp][c0 + reduce16_index(lane)] = red;
     }
     epi_sync();
@@ -464,7 +464,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           }
         }
       }
-      const float red = warp_reduce16<false>(acc, lane);
+      const float red = warp_reduce16<false, float>(acc, lane);
       if ((lane & 1) == 0) ms.wsum[warp][c0 + reduce16_index(lane)] = red;
     }
     epi_sync();
@@ -566,9 +566,69 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       epi_sync();
     }
 
-    // (h) mass of the sampling weights of each selected row over this CTA's slice; four
-    // sequences at a time so that their draft-logit loads are in flight together
-    if (ok) {
+    // (h) mass of the sampling weights of each selected row over this CTA's slice.
+    // Sample-only mode: every TMEM column is a selected row, so the tiles are read 16 columns
+    // (= 16 sequences) at a time, like the statistics passes.
+    if (ok && fp.sample_only) {
+#pragma unroll
+      for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+        if (c0 >= cp.B) break;
+        // A thread adds at most a handful of tiles per sequence, so its own partial sums stay in
+        // fp32 (32 double accumulators would not fit in registers); everything summed across
+        // lanes, warps and CTAs is double. The loop body is branch-free: with one warp per
+        // scheduler, branches around each sequence would serialise sixteen latency chains.
+        float sr[16], sp[16], lp2[16], lq2[16];
+        int kd[16];   // 0: residual, 1: p alone, 2: column past the last sequence
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int b = min(c0 + k, cp.B - 1);
+          sr[k] = 0.f; sp[k] = 0.f;
+          kd[k] = (c0 + k < cp.B) ? ms.sel_kind[b] : 2;
+          lp2[k] = ms.sel_lse_p[b] * kLog2e;
+          lq2[k] = ms.sel_lse_q[b] * kLog2e;
+        }
+        const int last_tile = fp.num_tiles - 1;
+        for (int i0 = 0; i0 < T; i0 += 2) {
+          const int vg0 = (t0 + i0) * kVocabTile + tid, vg1 = vg0 + kVocabTile;
+          const bool val0 = vg0 < V, val1 = (i0 + 1 < T) && vg1 < V;
+          // ws.w_sel holds the selected draft rows tile-major, [vocab tile][sequence][128]: this
+          // CTA's share is one contiguous block. Rows that need no residual were not gathered;
+          // what is read for them is discarded by the select below.
+          const float* base0 = ws.w_sel + ((size_t)(t0 + i0) * cp.B + min(c0, cp.B - 1)) * kVocabTile + tid;
+          const float* base1 = ws.w_sel + ((size_t)min(t0 + i0 + 1, last_tile) * cp.B + min(c0, cp.B - 1)) * kVocabTile + tid;
+          float d0[16], d1[16], v0[16], v1[16];
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const int kk = min(k, cp.B - 1 - min(c0, cp.B - 1));   // stay inside the buffer in a ragged last chunk
+            d0[k] = __ldg(base0 + kk * kVocabTile);
+            d1[k] = __ldg(base1 + kk * kVocabTile);
+          }
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, v0, v1);
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            const float p0 = fast_exp2(fmaf(v0[k], kLog2e, -lp2[k])), q0 = fast_exp2(fmaf(d0[k], kLog2e, -lq2[k]));
+            const float p1 = fast_exp2(fmaf(v1[k], kLog2e, -lp2[k])), q1 = fast_exp2(fmaf(d1[k], kLog2e, -lq2[k]));
+            const float r0 = kd[k] == 0 ? fmaxf(0.f, p0 - q0) : p0;
+            const float r1 = kd[k] == 0 ? fmaxf(0.f, p1 - q1) : p1;
+            const bool on0 = val0 && kd[k] < 2, on1 = val1 && kd[k] < 2;
+            sr[k] += (on0 ? r0 : 0.f) + (on1 ? r1 : 0.f);
+            sp[k] += (on0 ? p0 : 0.f) + (on1 ? p1 : 0.f);
+          }
+        }
+        double dsum[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) dsum[k] = (double)sr[k];
+        const double red_r = warp_reduce16<false, double>(dsum, lane);
+#pragma unroll
+        for (int k = 0; k < 16; ++k) dsum[k] = (double)sp[k];
+        const double red_p = warp_reduce16<false, double>(dsum, lane);
+        const int bq = c0 + reduce16_index(lane);
+        if ((lane & 1) == 0 && bq < cp.B) { ms.wd_r[bq][warp] = red_r; ms.wd_p[bq][warp] = red_p; }
+      }
+    }
+    // Full mode: the few selected rows sit in scattered columns; four sequences at a time so
+    // that their draft-logit loads are in flight together.
+    if (ok && !fp.sample_only) {
       for (int b0 = 0; b0 < cp.B; b0 += 4) {
         double sr[4] = {0.0, 0.0, 0.0, 0.0}, sp[4] = {0.0, 0.0, 0.0, 0.0};
         for (int i0 = 0; i0 < T; i0 += 8) {
@@ -659,14 +719,15 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             chunk += mc[u];
           }
         }
-        // exclusive prefix of the lane chunks, summed in lane order
-        double excl = 0.0, run = 0.0;
-        for (int l = 0; l < 32; ++l) {
-          const double cl = __shfl_sync(0xffffffffu, chunk, l);
-          if (l == lane) excl = run;
-          run += cl;
+        // exclusive prefix of the lane chunks (fixed-order warp scan, the same in every CTA)
+        double incl = chunk;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const double up = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += up;
         }
-        total = run;
+        const double excl = incl - chunk;
+        total = __shfl_sync(0xffffffffu, incl, 31);
         const double Tt = (double)ms.sel_u[b] * total;
         int owner = -1, last_mass = -1;
         double my_prefix = 0.0;
@@ -721,7 +782,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
-            dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
+            const float* src = fp.sample_only ? ws.w_sel + ((size_t)(t0 + i0 + u) * cp.B + b) * kVocabTile + tid
+                                              : dlrow + vg;
+            dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(src) : 0.f;
           }
           load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
 #pragma unroll

@@ -25,6 +25,7 @@ struct jd_handle_s {
   CUtensorMap tm_w;        // W as a [V, d] bf16 tensor, box 64 x 128, 128-byte swizzle
   CUtensorMap tm_w256;     // same tensor, box 64 x 256 (batched variant)
   cudaStream_t last_stream;
+  SideStream side;         // batched variant: draft statistics run next to the GEMM
   int last_variant;
   int last_launches;
   // device staging of the host-buffer entry point (allocated on first use)
@@ -186,6 +187,16 @@ jd_status_t jd_create(jd_handle_t* out, const jd_config_t* cfg) {
     delete h;
     return JD_ERR_CUDA;
   }
+  // the side stream is an optimisation: without it the batched variant runs its kernels in series
+  if (cudaStreamCreateWithFlags(&h->side.stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->side.fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->side.join, cudaEventDisableTiming) != cudaSuccess) {
+    cudaGetLastError();
+    if (h->side.stream) cudaStreamDestroy(h->side.stream);
+    if (h->side.fork) cudaEventDestroy(h->side.fork);
+    if (h->side.join) cudaEventDestroy(h->side.join);
+    h->side = SideStream{};
+  }
   *out = h;
   return JD_OK;
 }
@@ -194,6 +205,9 @@ jd_status_t jd_destroy(jd_handle_t h) {
   if (!h) return JD_OK;
   cudaSetDevice(h->cfg.device);
   cudaDeviceSynchronize();
+  if (h->side.stream) cudaStreamDestroy(h->side.stream);
+  if (h->side.fork) cudaEventDestroy(h->side.fork);
+  if (h->side.join) cudaEventDestroy(h->side.join);
   cudaFree(h->ws_base);
   cudaFree(h->st_H);
   cudaFree(h->st_x);
@@ -263,7 +277,7 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
         !make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)a->B, (uint64_t)c.d, (uint32_t)plan2.n_pad))
       return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
-    launches = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, a->H, h->w_judge, h->num_sms, st, &err);
+    launches = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, a->H, h->w_judge, h->num_sms, st, h->side, &err);
     if (launches < 0) return JD_ERR_CUDA;
   } else {
     CUtensorMap tm_h;

@@ -232,17 +232,30 @@ bool batched_supported(int dtype, int B, int d, int V, int num_sms) {
 
 int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
                 const CUtensorMap& tmH, const CUtensorMap& tmHsel, const void* H, const void* w_judge, int num_sms,
-                cudaStream_t st, cudaError_t* err) {
+                cudaStream_t st, const SideStream& side, cudaError_t* err) {
   const int R = cp.B * (cp.M + 1);
   const int np = (cp.V + kTileN - 1) / kTileN;
-  const int nq = launch_q_stats(cp, ws, st);
-  launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, st);
   const size_t smem = 1024 + kBMisc + (size_t)kBStages * (kAStage + kBStage);
   *err = cudaFuncSetAttribute(gemm_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (*err != cudaSuccess) return -1;
   const int row_blocks = (R + kTileM - 1) / kTileM, voc_blocks = np;
   const int grid = std::min(num_sms, row_blocks * voc_blocks);
-  gemm_stats_kernel<<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+  int nq;
+  if (side.stream) {
+    // The draft statistics (HBM-bound) and the judge dots do not depend on the GEMM (tensor-bound):
+    // they run on the handle's side stream next to it and join before the decision.
+    if ((*err = cudaEventRecord(side.fork, st)) != cudaSuccess) return -1;
+    gemm_stats_kernel<<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+    if ((*err = cudaStreamWaitEvent(side.stream, side.fork, 0)) != cudaSuccess) return -1;
+    nq = launch_q_stats(cp, ws, side.stream);
+    launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, side.stream);
+    if ((*err = cudaEventRecord(side.join, side.stream)) != cudaSuccess) return -1;
+    if ((*err = cudaStreamWaitEvent(st, side.join, 0)) != cudaSuccess) return -1;
+  } else {
+    nq = launch_q_stats(cp, ws, st);
+    launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, st);
+    gemm_stats_kernel<<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+  }
   launch_decide(cp, ws, np, nq, st);
   gather_rows_kernel<<<dim3(cp.B, 8), 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H);
   FusedPlan plan;

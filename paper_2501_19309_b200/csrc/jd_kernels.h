@@ -36,9 +36,14 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
 // Two-pass tensor-core variant for many rows (jd_batched_sm100.cu). tmW256 / tmW128: W with
 // 256- and 128-row boxes; tmH: H with a 128-row box; tmHsel: the handle's [B, d] gather buffer
 // with the fused plan's box. Returns the number of kernels launched, or -1 with *err set.
+// Optional second stream of a handle (with the two events that fork to it and join from it).
+struct SideStream {
+  cudaStream_t stream;
+  cudaEvent_t fork, join;
+};
 bool batched_supported(int dtype, int B, int d, int V, int num_sms);
 int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
                 const CUtensorMap& tmH, const CUtensorMap& tmHsel, const void* H, const void* w_judge, int num_sms,
-                cudaStream_t st, cudaError_t* err);
+                cudaStream_t st, const SideStream& side, cudaError_t* err);
 
 }  // namespace jd

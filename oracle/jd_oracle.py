@@ -23,6 +23,14 @@ Sec. 4.1 "Inference"; 0-indexed here, the paper is 1-indexed):
               from p_M after a fully accepted block; inverse CDF in ascending
               token id with one uniform.
 
+Deterministic variants of the standard test (Sec. 3.2 speaks of acceptance "under greedy
+decoding"; Sec. 5.1 "Training-free baseline" defines top-K verification): with rule="topk" the
+candidate x_j passes the standard test iff it is among the K highest-valued entries of p_j
+(K = 1 is greedy verification, K = V accepts everything), and the next token is the target's
+greedy token argmax p_a, at a rejection as well as after a fully accepted block. No uniform is
+drawn and the draft distribution plays no role. Equal logits are ordered by token id (lower id
+ranks higher), so "among the K highest" and "argmax" are unique.
+
 Readings taken where the paper is silent (all restated in the design notes):
   * the judge for draft token j reads row j+1 of H, the embedding produced by
     feeding that token (Sec. 4.1 speaks of the embedding of the current token);
@@ -60,6 +68,8 @@ import numpy as np
 MODE_STANDARD, MODE_JUDGE, MODE_JUDGE_OR_STANDARD = 0, 1, 2
 RESAMPLE_RESIDUAL, RESAMPLE_TARGET_P = 0, 1
 STREAM_ACCEPT, STREAM_SAMPLE = 0, 1
+
+RULE_SAMPLING, RULE_TOPK = 0, 1
 
 _MODES = {"standard": MODE_STANDARD, "judge": MODE_JUDGE, "judge_or_standard": MODE_JUDGE_OR_STANDARD}
 _RESAMPLE = {"residual": RESAMPLE_RESIDUAL, "target_p": RESAMPLE_TARGET_P}
@@ -179,7 +189,8 @@ class OracleResult:
     u_sample: np.ndarray            # [B] float64 uniform of the token draw
     margin_accept: np.ndarray       # [B, M] |u - min(1, p/q)|
     margin_judge: np.ndarray        # [B, M] |s - tau|
-    margin_cdf: np.ndarray          # [B] distance of T to the nearest CDF edge of the token, / sum(r)
+    margin_cdf: np.ndarray          # [B] distance of T to the nearest CDF edge of the token, / sum(r);
+                                    #     rule "topk": gap between the two largest logits of row a, scaled
     sample_T: np.ndarray            # [B] T = u' * sum(r)
     sample_mass: np.ndarray         # [B] sum(r)
     sample_weights: dict            # b -> r[V] float64 (un-normalised sampling weights)
@@ -193,16 +204,27 @@ class OracleResult:
         return lo, float(cdf[token])
 
 
+def rank_in_row(row: np.ndarray, x: int) -> int:
+    """Position of token x when the row is sorted by value, highest first, equal values by
+    ascending token id: the number of entries that rank above x."""
+    lx = row[x]
+    return int(np.count_nonzero(row > lx) + np.count_nonzero(row[:x] == lx))
+
+
 def jd_oracle_verify(W, w_judge, b_judge: float, H, draft_tokens, draft_logits, tau: float,
                      seed: int, mode="judge_or_standard", resample="residual",
                      sequences: Optional[Sequence[int]] = None, keep_logits: bool = False,
                      u_accept: Optional[np.ndarray] = None,
-                     u_sample: Optional[np.ndarray] = None) -> OracleResult:
+                     u_sample: Optional[np.ndarray] = None,
+                     rule="sampling", top_k: int = 1) -> OracleResult:
     """One verification call, step by step, in float64.
 
     ``u_accept`` [B, M] / ``u_sample`` [B], when given, replace the Philox
     uniforms (used by the enumeration tests, which sweep u over a dyadic grid).
     ``sequences`` restricts the work to some b (sampled checks at full size)."""
+    rule = {"sampling": RULE_SAMPLING, "greedy": RULE_TOPK, "topk": RULE_TOPK}[rule] if isinstance(rule, str) else int(rule)
+    if rule == RULE_TOPK and top_k < 1:
+        raise ValueError("top_k must be >= 1")
     mode = _MODES[mode] if isinstance(mode, str) else int(mode)
     resample = _RESAMPLE[resample] if isinstance(resample, str) else int(resample)
     H = np.asarray(H)
@@ -241,20 +263,50 @@ def jd_oracle_verify(W, w_judge, b_judge: float, H, draft_tokens, draft_logits, 
             xj = int(x[b, j])
             P = float(np.exp(L[j, xj] - lse_p[j]))                          # p_j[x_j]
             Q = float(np.exp(dlj[xj] - lse_q[j]))                           # q_j[x_j]
-            u = float(u_accept[b, j]) if u_accept is not None else uniform24(seed, b, j, STREAM_ACCEPT)
-            z_std = int(u * Q < P)                                          # (Eq. 4)
+            if rule == RULE_TOPK:
+                u = float("nan")
+                z_std = int(rank_in_row(L[j], xj) < top_k)                  # among the K highest of p_j
+            else:
+                u = float(u_accept[b, j]) if u_accept is not None else uniform24(seed, b, j, STREAM_ACCEPT)
+                z_std = int(u * Q < P)                                      # (Eq. 4)
             s = sigmoid(float(wj @ Hb[j + 1]) + b_judge)                    # judge on x_j's embedding
             z_judge = int(s > tau)                                          # (Sec. 4.1)
             z.append(combine_masks(z_std, z_judge, mode))
             res.p_draft[b, j], res.q_draft[b, j], res.judge_scores[b, j] = P, Q, s
             res.masks[b, j] = z_std | (z_judge << 1)
             res.u_accept[b, j] = u
-            ratio = 1.0 if Q == 0.0 else min(1.0, P / Q)
-            res.margin_accept[b, j] = abs(u - ratio)
+            if rule == RULE_TOPK:
+                # distance of the candidate's logit to the value it would have to cross, in units
+                # of the row's logit scale
+                srt = np.sort(L[j])[::-1]
+                scale = max(abs(float(srt[0])), float(np.sqrt(np.mean(L[j] * L[j]))))
+                if z_std:
+                    edge = float(srt[top_k]) if top_k < V else -np.inf
+                    res.margin_accept[b, j] = (float(L[j, xj]) - edge) / scale
+                else:
+                    res.margin_accept[b, j] = (float(srt[top_k - 1]) - float(L[j, xj])) / scale
+            else:
+                ratio = 1.0 if Q == 0.0 else min(1.0, P / Q)
+                res.margin_accept[b, j] = abs(u - ratio)
             res.margin_judge[b, j] = abs(s - tau)
 
         a = accepted_prefix_length(z)                                       # prefix rule
         res.accept_len[b] = a
+
+        if rule == RULE_TOPK:
+            # the target's greedy token, at a rejection and after a fully accepted block alike
+            t = int(np.argmax(L[a]))                                        # first index among equal maxima
+            res.next_token[b] = t
+            top2 = np.partition(L[a], -2)[-2:] if V > 1 else np.array([L[a, t], L[a, t]])
+            scale = max(abs(float(L[a, t])), float(np.sqrt(np.mean(L[a] * L[a]))))
+            res.margin_cdf[b] = float(top2[1] - top2[0]) / scale
+            w1 = np.zeros(V)
+            w1[t] = 1.0
+            res.sample_weights[b] = w1
+            res.sample_T[b], res.sample_mass[b] = 0.0, 1.0
+            if keep_logits:
+                res.logits[b] = L
+            continue
 
         p_a = np.exp(L[a] - lse_p[a])
         if a < M and resample == RESAMPLE_RESIDUAL:

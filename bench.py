@@ -36,9 +36,10 @@ METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes (read + write) per launch of the fused kernel from an ncu capture, per workload;
-# None until captured for the kernel as it stands.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes (read + write) per verification call from the ncu captures summarised under profiles/
+# (dominant kernels of each workload); set an entry to None when its kernel changes.
+NCU_TRAFFIC_BYTES = {"cfg1-8B-head": 1.0587e9, "cfg2-70B-head": 2.1758e9, "cfg3-405B-head": 4.2329e9,
+                     "cfg4-batched": 2.149e9 + 2.152e9}   # cfg4: GEMM pass + second pass
 VARIANT_NAMES = {1: "simt", 2: "fused", 3: "batched"}
 
 

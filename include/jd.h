@@ -66,9 +66,10 @@ typedef enum {
   JD_VARIANT_AUTO = 0,
   JD_VARIANT_SIMT = 1,   /* CUDA-core reference pipeline: any shape, f32 or bf16 */
   JD_VARIANT_FUSED = 2,  /* one persistent tcgen05/TMA kernel, logits parked in tensor memory;
-                            bf16, d % 64 == 0, B*(M+1) <= 80, V <= 7*128*(number of SMs) */
+                            bf16, d % 64 == 0, B*(M+1) <= 96, V small enough for every CTA to
+                            keep its vocabulary tiles on chip (128256 fits on 148 SMs) */
   JD_VARIANT_BATCHED = 3 /* tcgen05 GEMM with fused statistics + second pass over the selected
-                            rows; bf16, d % 64 == 0, any number of rows */
+                            rows; bf16, d % 64 == 0, any number of rows, B <= 96 */
 } jd_variant_t;
 
 typedef struct {

@@ -61,6 +61,16 @@ typedef enum { JD_MODE_STANDARD = 0, JD_MODE_JUDGE = 1, JD_MODE_JUDGE_OR_STANDAR
  * After a fully accepted block the token always comes from p_M. */
 typedef enum { JD_RESAMPLE_RESIDUAL = 0, JD_RESAMPLE_TARGET_P = 1 } jd_resample_t;
 
+/* How the standard (non-judge) test decides, and how the next token is chosen.
+ * SAMPLING: the stochastic test of Eq. 4 with the residual / bonus draw described above.
+ * TOPK:     deterministic verification: the candidate passes iff it is among the top_k highest-valued
+ *           entries of p_j (Sec. 5.1 "Training-free baseline"); top_k = 1 is greedy verification
+ *           (acceptance "under greedy decoding", Sec. 3.2), top_k = V accepts everything. The next
+ *           token is the target's greedy token argmax p_a, at a rejection and after a full block.
+ *           Equal logits rank by token id (lower id first). No uniform is drawn; the draft logits
+ *           only feed the q_draft output. */
+typedef enum { JD_RULE_SAMPLING = 0, JD_RULE_TOPK = 1 } jd_rule_t;
+
 /* Kernel family used by jd_verify. AUTO picks the fastest one that supports the shape. */
 typedef enum {
   JD_VARIANT_AUTO = 0,
@@ -94,6 +104,8 @@ typedef struct {
   int32_t mode;                /* jd_mode_t */
   int32_t resample;            /* jd_resample_t */
   int32_t variant;             /* jd_variant_t; JD_VARIANT_AUTO in production */
+  int32_t rule;                /* jd_rule_t */
+  int32_t top_k;               /* K of JD_RULE_TOPK, >= 1; ignored by JD_RULE_SAMPLING */
   /* outputs, always written */
   int32_t* accept_len;         /* [B] number of accepted draft tokens, 0..M */
   int32_t* next_token;         /* [B] the corrected (accept_len < M) or bonus (== M) token */
@@ -171,7 +183,7 @@ jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* s
  * allocating call is made here.
  *   d, V, W, w_judge, b_judge : the head, as for jd_set_head (device pointers, 16-byte aligned)
  *   args                     : as for jd_verify (device pointers); variant must be AUTO or FUSED,
- *                              logits_debug NULL
+ *                              rule JD_RULE_SAMPLING, logits_debug NULL
  *   device_status            : optional device pointer to one uint32 that receives the call's
  *                              device status (JD_OK, JD_ERR_TIMEOUT, JD_ERR_BAD_TOKEN); NULL to skip
  * The call uses the CURRENT device. Its first call on a device looks up the array's device

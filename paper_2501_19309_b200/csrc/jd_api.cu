@@ -112,6 +112,9 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
   w.w_sel = (float*)take(maxB * (((size_t)c.V + kVocabTile - 1) / kVocabTile * kVocabTile) * 4);
   w.p_sel = (float*)take(maxB * (size_t)c.V * 4);
   w.h_sel = (__nv_bfloat16*)take(maxB * (size_t)c.d * 2);
+  w.cnt = (int*)take(maxR * 4);
+  w.argidx = (int*)take(maxR * 4);
+  w.part_idx = (int*)take(maxR * np * 4);
   w.status = (unsigned*)take(256);
   w.barrier = (unsigned*)take(256);
   w.np_cap = (int)np;
@@ -134,6 +137,8 @@ jd_status_t validate(jd_handle_t h, const jd_verify_args_t* a) {
   if (a->mode < JD_MODE_STANDARD || a->mode > JD_MODE_JUDGE_OR_STANDARD) return JD_ERR_INVALID_ARG;
   if (a->resample < JD_RESAMPLE_RESIDUAL || a->resample > JD_RESAMPLE_TARGET_P) return JD_ERR_INVALID_ARG;
   if (a->variant < JD_VARIANT_AUTO || a->variant > JD_VARIANT_BATCHED) return JD_ERR_INVALID_ARG;
+  if (a->rule != JD_RULE_SAMPLING && a->rule != JD_RULE_TOPK) return JD_ERR_INVALID_ARG;
+  if (a->rule == JD_RULE_TOPK && a->top_k < 1) return JD_ERR_INVALID_ARG;
   return JD_OK;
 }
 
@@ -245,6 +250,7 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   cp.draft_logits = a->draft_logits;
   cp.tau = a->tau; cp.b_judge = h->b_judge; cp.seed = a->seed;
   cp.mode = a->mode; cp.resample = a->resample;
+  cp.rule = a->rule; cp.top_k = a->top_k;
   cp.accept_len = a->accept_len; cp.next_token = a->next_token;
   cp.judge_scores = a->judge_scores; cp.p_draft = a->p_draft;
   cp.q_draft = a->q_draft; cp.masks = a->masks;
@@ -266,6 +272,11 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   if (cudaSetDevice(c.device) != cudaSuccess) return JD_ERR_CUDA;
   // status word and the grid-barrier counters behind it start every call at zero
   if (cudaMemsetAsync(h->ws.status, 0, 512, st) != cudaSuccess) return JD_ERR_CUDA;
+  if (a->rule == JD_RULE_TOPK) {   // rank counters start at zero, argmax candidates at a large id
+    if (cudaMemsetAsync(h->ws.cnt, 0, (size_t)R * 4, st) != cudaSuccess ||
+        cudaMemsetAsync(h->ws.argidx, 0x7F, (size_t)R * 4, st) != cudaSuccess)
+      return JD_ERR_CUDA;
+  }
   int launches = 0;
   if (variant == JD_VARIANT_SIMT) {
     launches = run_simt(cp, h->ws, h->W, h->w_judge, a->H, c.dtype, a->logits_debug, st);

@@ -50,6 +50,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// kCount == false: softmax statistics + gather (first pass).
+// kCount == true : top-K rule, after the fold: the same GEMM again (bit-identical logits), the
+//                  epilogue counts the entries that rank above the drafted token and records the
+//                  lowest token id equal to the folded row maximum.
+template <bool kCount>
 __global__ void __launch_bounds__(kBThreads, 1)
 gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, CallParams cp,
                   Workspace ws, int R, int np) {
@@ -153,6 +158,12 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       tc_fence_after();
       float m = -INFINITY, s = 0.f, g = 0.f;
       bool have_g = false;
+      int above = 0, cand = 0x7F7F7F7F;
+      float g_ref = 0.f, rmax = 0.f;
+      if (kCount && row < R) {
+        rmax = ws.row_max[row];
+        if (x >= 0) g_ref = ws.gath[row];
+      }
 #pragma unroll 1
       for (int c0 = 0; c0 < kTileN; c0 += 32) {
         float v[32];
@@ -161,6 +172,15 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         if (nvalid < 32) {
 #pragma unroll
           for (int k = 0; k < 32; ++k) if (k >= nvalid) v[k] = -INFINITY;
+        }
+        if (kCount) {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) {
+            const int col = v0 + c0 + k;
+            if (x >= 0 && (v[k] > g_ref || (v[k] == g_ref && col < x))) ++above;
+            if (v[k] == rmax) cand = min(cand, col);
+          }
+          continue;
         }
         float cm = v[0];
 #pragma unroll
@@ -184,9 +204,14 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       epi_sync();
       if (tid == 0) mbar_arrive(smem_u32(&ms.tmem_empty[buf]));
       if (row < R) {
-        ws.part_max[(size_t)row * np + vb] = m;
-        ws.part_sum[(size_t)row * np + vb] = s;
-        if (have_g) ws.gath[row] = g;
+        if (kCount) {
+          if (above) atomicAdd(ws.cnt + row, above);
+          if (cand != 0x7F7F7F7F) atomicMin(ws.argidx + row, cand);
+        } else {
+          ws.part_max[(size_t)row * np + vb] = m;
+          ws.part_sum[(size_t)row * np + vb] = s;
+          if (have_g) ws.gath[row] = g;
+        }
       }
     }
     if (!ok && tid == 0) set_status(ws.status, JD_ERR_TIMEOUT);
@@ -236,7 +261,9 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
   const int R = cp.B * (cp.M + 1);
   const int np = (cp.V + kTileN - 1) / kTileN;
   const size_t smem = 1024 + kBMisc + (size_t)kBStages * (kAStage + kBStage);
-  *err = cudaFuncSetAttribute(gemm_stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  *err = cudaFuncSetAttribute(gemm_stats_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (*err == cudaSuccess)
+    *err = cudaFuncSetAttribute(gemm_stats_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (*err != cudaSuccess) return -1;
   const int row_blocks = (R + kTileM - 1) / kTileM, voc_blocks = np;
   const int grid = std::min(num_sms, row_blocks * voc_blocks);
@@ -245,7 +272,7 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
     // The draft statistics (HBM-bound) and the judge dots do not depend on the GEMM (tensor-bound):
     // they run on the handle's side stream next to it and join before the decision.
     if ((*err = cudaEventRecord(side.fork, st)) != cudaSuccess) return -1;
-    gemm_stats_kernel<<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+    gemm_stats_kernel<false><<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
     if ((*err = cudaStreamWaitEvent(side.stream, side.fork, 0)) != cudaSuccess) return -1;
     nq = launch_q_stats(cp, ws, side.stream);
     launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, side.stream);
@@ -254,9 +281,15 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
   } else {
     nq = launch_q_stats(cp, ws, st);
     launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, st);
-    gemm_stats_kernel<<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+    gemm_stats_kernel<false><<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
   }
-  launch_decide(cp, ws, np, nq, st);
+  launch_fold(cp, ws, np, nq, st);
+  if (cp.rule == JD_RULE_TOPK) {   // second GEMM pass for ranks and argmax; no token draw
+    gemm_stats_kernel<true><<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+    launch_decide(cp, ws, st);
+    return 6;
+  }
+  launch_decide(cp, ws, st);
   gather_rows_kernel<<<dim3(cp.B, 8), 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H);
   FusedPlan plan;
   if (!fused_supported(JD_DTYPE_BF16, cp.B, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }

@@ -38,6 +38,9 @@ struct Workspace {
   float* w_sel;        // [maxB][V]  sampling weights (SIMT variant); in the batched variant the selected
                        //            draft rows, tile-major [ceil(V/128)][B][128]
   float* p_sel;        // [maxB][V]  p of the selected row (same)
+  int* cnt;            // [maxR] top-K rule: entries of the row that rank above the drafted token
+  int* argidx;         // [maxR] top-K rule: lowest token id that attains the row maximum
+  int* part_idx;       // [maxR][np] top-K rule, fused variant: per-CTA argmax candidates
   __nv_bfloat16* h_sel;  // [maxB][d] selected rows of H gathered for the batched variant's second pass
   unsigned* status;    // [1] device status word (jd_status_t of the first device-side problem)
   unsigned* barrier;   // [8] grid-barrier counters of the fused variant
@@ -117,6 +120,7 @@ struct CallParams {
   float tau, b_judge;
   uint64_t seed;
   int mode, resample;
+  int rule, top_k;
   int32_t* accept_len;
   int32_t* next_token;
   float* judge_scores;
@@ -147,7 +151,7 @@ __device__ __forceinline__ int decide_sequence(const CallParams& cp, const Works
       const float P = expf(__ldcg(ws.gath + row) - ws.row_lse[row]);
       const float Q = expf(__ldcg(ws.qgath + bm) - ws.q_lse[bm]);
       const float u = philox_uniform(cp.seed, b, j, 0);
-      const bool z_std = (u * Q < P);
+      const bool z_std = (cp.rule == JD_RULE_TOPK) ? (__ldcg(ws.cnt + row) < cp.top_k) : (u * Q < P);
       const float s = 1.0f / (1.0f + expf(-(__ldcg(ws.judge_logit + bm) + cp.b_judge)));
       const bool z_judge = (s > cp.tau);
       ok = cp.mode == JD_MODE_STANDARD ? z_std : (cp.mode == JD_MODE_JUDGE ? z_judge : (z_std || z_judge));
@@ -166,11 +170,15 @@ __device__ __forceinline__ int decide_sequence(const CallParams& cp, const Works
     const int row = b * (M + 1) + a;
     ws.sel_row[b] = row;
     const bool residual = (a < M) && (cp.resample == JD_RESAMPLE_RESIDUAL);
-    ws.sel_kind[b] = residual ? 0 : 1;
+    ws.sel_kind[b] = (cp.rule == JD_RULE_TOPK) ? 2 : (residual ? 0 : 1);   // 2: greedy token, nothing to draw
     ws.sel_lse_p[b] = ws.row_lse[row];
     ws.sel_lse_q[b] = residual ? ws.q_lse[b * M + a] : 0.f;
     ws.sel_u[b] = philox_uniform(cp.seed, b, a, 1);
-    if (write_outputs) cp.accept_len[b] = a;
+    if (write_outputs) {
+      cp.accept_len[b] = a;
+      // top-K rule: the next token is the row's argmax, known already unless the caller folds it later
+      if (cp.rule == JD_RULE_TOPK && ws.argidx) cp.next_token[b] = __ldcg(ws.argidx + row);
+    }
   }
   return a;
 }

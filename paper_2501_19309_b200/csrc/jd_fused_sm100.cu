@@ -485,6 +485,59 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     epi_sync();
     ok = (*abort_flag == 0);
 
+    // (f0) top-K rule: over the parked tiles, count the entries of every draft row that rank above
+    // the drafted token (its logit is known grid-wide since barrier 1) and note the lowest token id
+    // that attains this CTA's row maximum. Counts go to global counters with integer atomics
+    // (order-independent), the argmax candidates beside the per-CTA maxima.
+    if (ok && cp.rule == JD_RULE_TOPK) {
+      int* wcnt = reinterpret_cast<int*>(&ms.wmax[0][0]);   // the float statistics have been written out
+      int* widx = reinterpret_cast<int*>(&ms.wsum[0][0]);
+#pragma unroll
+      for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+        float gref[16], cmx[16];
+        int xr[16], cnt[16], neg[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const int r = c0 + k;
+          xr[k] = ms.x_row[r];
+          gref[k] = (r < R && xr[k] >= 0) ? __ldcg(ws.gath + r) : INFINITY;   // nothing ranks above +inf
+          cmx[k] = ms.cta_max[r];
+          cnt[k] = 0;
+          neg[k] = -0x7F7F7F7F;
+        }
+        for (int i0 = 0; i0 < T; i0 += 2) {
+          float v0[16], v1[16];
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, v0, v1);
+          const int vg0 = (t0 + i0) * kVocabTile + tid, vg1 = vg0 + kVocabTile;
+          const bool val0 = vg0 < V, val1 = (i0 + 1 < T) && vg1 < V;
+#pragma unroll
+          for (int k = 0; k < 16; ++k) {
+            if (val0) {
+              cnt[k] += (v0[k] > gref[k] || (v0[k] == gref[k] && vg0 < xr[k])) ? 1 : 0;
+              if (v0[k] == cmx[k]) neg[k] = max(neg[k], -vg0);
+            }
+            if (val1) {
+              cnt[k] += (v1[k] > gref[k] || (v1[k] == gref[k] && vg1 < xr[k])) ? 1 : 0;
+              if (v1[k] == cmx[k]) neg[k] = max(neg[k], -vg1);
+            }
+          }
+        }
+        const int red_c = warp_reduce16<false, int>(cnt, lane);
+        const int red_i = warp_reduce16<true, int>(neg, lane);
+        if ((lane & 1) == 0) {
+          wcnt[warp * N_PAD + c0 + reduce16_index(lane)] = red_c;
+          widx[warp * N_PAD + c0 + reduce16_index(lane)] = red_i;
+        }
+      }
+      epi_sync();
+      if (tid < R) {
+        const int c = (wcnt[tid] + wcnt[N_PAD + tid]) + (wcnt[2 * N_PAD + tid] + wcnt[3 * N_PAD + tid]);
+        const int i = max(max(widx[tid], widx[N_PAD + tid]), max(widx[2 * N_PAD + tid], widx[3 * N_PAD + tid]));
+        if (c > 0 && ms.x_row[tid] >= 0) atomicAdd(ws.cnt + tid, c);
+        ws.part_idx[(size_t)tid * G + cta] = -i;
+      }
+    }
+
     // (f) fold the per-CTA statistics: the R target rows and the B*M draft rows are dealt out
     // over the grid, one per warp, so that no CTA reads more than a few rows' worth of partials
     if (ok) {
@@ -550,6 +603,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       lw.sel_lse_p = ms.sel_lse_p;
       lw.sel_lse_q = ms.sel_lse_q;
       lw.sel_u = ms.sel_u;
+      lw.argidx = nullptr;   // top-K rule: the next token is folded below, not read from global
       for (int b = warp; b < cp.B; b += 4) decide_sequence(cp, lw, b, cta == 0);
     }
     epi_sync();
@@ -566,10 +620,37 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       epi_sync();
     }
 
+    // top-K rule: the next token is the argmax of the selected row; CTA 0 folds the per-CTA maxima
+    // and their candidates (larger value first, then lower token id). Nothing is drawn.
+    const bool draw = (cp.rule != JD_RULE_TOPK);
+    if (ok && !draw && cta == 0) {
+      for (int b = warp; b < cp.B; b += 4) {
+        const int row = ms.sel_row[b];
+        float bm = -INFINITY;
+        int bi = 0x7F7F7F7F;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int c = lane + 32 * u;
+          if (c < G) {
+            const float m = __ldcg(ws.part_max + (size_t)row * G + c);
+            const int i = __ldcg(ws.part_idx + (size_t)row * G + c);
+            if (m > bm || (m == bm && i < bi)) { bm = m; bi = i; }
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float m = __shfl_xor_sync(0xffffffffu, bm, o);
+          const int i = __shfl_xor_sync(0xffffffffu, bi, o);
+          if (m > bm || (m == bm && i < bi)) { bm = m; bi = i; }
+        }
+        if (lane == 0) cp.next_token[b] = bi;
+      }
+    }
+
     // (h) mass of the sampling weights of each selected row over this CTA's slice.
     // Sample-only mode: every TMEM column is a selected row, so the tiles are read 16 columns
     // (= 16 sequences) at a time, like the statistics passes.
-    if (ok && fp.sample_only) {
+    if (ok && draw && fp.sample_only) {
 #pragma unroll
       for (int c0 = 0; c0 < N_PAD; c0 += 16) {
         if (c0 >= cp.B) break;
@@ -628,7 +709,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     // Full mode: the few selected rows sit in scattered columns; four sequences at a time so
     // that their draft-logit loads are in flight together.
-    if (ok && !fp.sample_only) {
+    if (ok && draw && !fp.sample_only) {
       for (int b0 = 0; b0 < cp.B; b0 += 4) {
         double sr[4] = {0.0, 0.0, 0.0, 0.0}, sp[4] = {0.0, 0.0, 0.0, 0.0};
         for (int i0 = 0; i0 < T; i0 += 8) {
@@ -675,7 +756,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
     }
     epi_sync();
-    if (ok && tid < cp.B) {
+    if (ok && draw && tid < cp.B) {
       ws.mass_r[(size_t)tid * G + cta] = (ms.wd_r[tid][0] + ms.wd_r[tid][1]) + (ms.wd_r[tid][2] + ms.wd_r[tid][3]);
       ws.mass_p[(size_t)tid * G + cta] = (ms.wd_p[tid][0] + ms.wd_p[tid][1]) + (ms.wd_p[tid][2] + ms.wd_p[tid][3]);
     }
@@ -683,7 +764,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     epi_sync();
 
     // ------------------------------------------------------------------ grid barrier 3
-    if (tid == 0) {
+    if (tid == 0 && draw) {
       if (!ok || !grid_arrive_and_wait(ws.barrier + 2, (unsigned)G, abort_flag)) {
         *abort_flag = 1;
         set_status(ws.status, JD_ERR_TIMEOUT);
@@ -694,7 +775,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
     // (i) inverse CDF in ascending token id. First, one warp per sequence finds the CTA whose
     // slice contains T = u * total (same arithmetic in every CTA, so every CTA agrees) ...
-    if (ok) {
+    if (ok && draw) {
       const int per = (G + 31) / 32;   // lane l owns CTAs [l*per, (l+1)*per), per <= 8
       for (int b = warp; b < cp.B; b += 4) {
         const double* mass = ws.mass_r + (size_t)b * G;
@@ -765,7 +846,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     epi_sync();
     // ... then the owning CTA finds the tile from the tile masses and the token inside that tile
-    if (ok) {
+    if (ok && draw) {
       for (int b = 0; b < cp.B; ++b) {
         if (ms.own_cta[b] != cta) continue;
         const int row = ms.sel_row[b];

@@ -12,7 +12,8 @@ int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const voi
              float* logits_debug, cudaStream_t st);
 int launch_q_stats(const CallParams& cp, const Workspace& ws, cudaStream_t st);   // returns partials per draft row
 void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, const void* w, int dtype, cudaStream_t st);
-void launch_decide(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st);   // fold + decide: 2 launches
+void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st);
+void launch_decide(const CallParams& cp, const Workspace& ws, cudaStream_t st);
 void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream_t st);
 void launch_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot, const int32_t* stream, int n,
                             float* out, cudaStream_t st);

@@ -9,14 +9,18 @@ namespace jd {
 
 // -----------------------------------------------------------------------------------------
 // Stage 1: logits of a [128 vocab] x [16 rows] tile by smem-tiled FMA.
-//   kSample == false: per-(row, vocab tile) softmax partials + gather of L[row, x_j]
-//   kSample == true : rows are the selected rows (one per sequence); writes the sampling
-//                     weights and p of that row plus their per-tile masses
+//   kMode 0: per-(row, vocab tile) softmax partials + gather of L[row, x_j]
+//   kMode 1: rows are the selected rows (one per sequence); writes the sampling weights and p
+//            of that row plus their per-tile masses
+//   kMode 2: top-K rule, after the fold: counts the entries of every row that rank above the
+//            drafted token and records the lowest token id that attains the row maximum. The
+//            logits are recomputed with the same instruction sequence as in mode 0, so they are
+//            bit-identical to the gathered logit and to the folded maximum.
 // -----------------------------------------------------------------------------------------
 constexpr int kSimtRows = 16;
 constexpr int kSimtK = 32;
 
-template <typename T, bool kSample>
+template <typename T, int kMode>
 __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, Workspace ws, const T* __restrict__ W,
                                                                  const T* __restrict__ H, int R, int np,
                                                                  float* __restrict__ logits_debug) {
@@ -26,6 +30,7 @@ __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, 
   __shared__ double s_d[2][4][kSimtRows];
   __shared__ int s_row[kSimtRows];
 
+  constexpr bool kSample = (kMode == 1);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = blockIdx.x;
   const int v = tile * kVocabTile + tid;
@@ -71,7 +76,24 @@ __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, 
   }
 
   const bool valid_v = v < V;
-  if (!kSample) {
+  if (kMode == 2) {
+#pragma unroll
+    for (int i = 0; i < kSimtRows; ++i) {
+      const int row = s_row[i];
+      bool above = false;
+      if (row >= 0) {
+        const int b = row / (cp.M + 1), j = row % (cp.M + 1);
+        if (valid_v && acc[i] == ws.row_max[row]) atomicMin(ws.argidx + row, v);
+        if (j < cp.M && valid_v) {
+          const int x = min(max(cp.draft_tokens[b * cp.M + j], 0), V - 1);
+          const float g = ws.gath[row];
+          above = acc[i] > g || (acc[i] == g && v < x);
+        }
+      }
+      const unsigned mask = __ballot_sync(0xffffffffu, above);
+      if (lane == 0 && mask) atomicAdd(ws.cnt + row, __popc(mask));
+    }
+  } else if (!kSample) {
 #pragma unroll
     for (int i = 0; i < kSimtRows; ++i) {
       const int row = s_row[i];
@@ -321,9 +343,12 @@ void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, cons
     judge_dot_kernel<float><<<cp.B * cp.M, 256, 0, st>>>(cp, ws, (const float*)H, (const float*)w);
 }
 
-void launch_decide(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st) {
+void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st) {
   const int items = cp.B * (2 * cp.M + 1);
   fold_stats_kernel<<<(items + 7) / 8, 256, 0, st>>>(cp, ws, np, nq);
+}
+
+void launch_decide(const CallParams& cp, const Workspace& ws, cudaStream_t st) {
   decide_kernel<<<(cp.B + 3) / 4, 128, 0, st>>>(cp, ws);
 }
 
@@ -332,26 +357,37 @@ void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream
 }
 
 template <typename T>
-static void simt_logits(const CallParams& cp, const Workspace& ws, const void* W, const void* H, bool sample, int np,
+static void simt_logits(const CallParams& cp, const Workspace& ws, const void* W, const void* H, int mode, int np,
                         float* logits_debug, cudaStream_t st) {
-  const int R = sample ? cp.B : cp.B * (cp.M + 1);
+  const int R = mode == 1 ? cp.B : cp.B * (cp.M + 1);
   dim3 grid(np, (R + kSimtRows - 1) / kSimtRows);
-  if (sample)
-    simt_logits_kernel<T, true><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, nullptr);
+  if (mode == 1)
+    simt_logits_kernel<T, 1><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, nullptr);
+  else if (mode == 2)
+    simt_logits_kernel<T, 2><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, nullptr);
   else
-    simt_logits_kernel<T, false><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, logits_debug);
+    simt_logits_kernel<T, 0><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, logits_debug);
 }
 
 int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const void* w_judge, const void* H, int dtype,
              float* logits_debug, cudaStream_t st) {
   const int np = (cp.V + kVocabTile - 1) / kVocabTile;
+  const bool bf = dtype == JD_DTYPE_BF16;
+  auto logits = [&](int mode, float* dbg) {
+    if (bf) simt_logits<__nv_bfloat16>(cp, ws, W, H, mode, np, dbg, st);
+    else simt_logits<float>(cp, ws, W, H, mode, np, dbg, st);
+  };
   const int nq = launch_q_stats(cp, ws, st);
   launch_judge(cp, ws, H, w_judge, dtype, st);
-  if (dtype == JD_DTYPE_BF16) simt_logits<__nv_bfloat16>(cp, ws, W, H, false, np, logits_debug, st);
-  else simt_logits<float>(cp, ws, W, H, false, np, logits_debug, st);
-  launch_decide(cp, ws, np, nq, st);
-  if (dtype == JD_DTYPE_BF16) simt_logits<__nv_bfloat16>(cp, ws, W, H, true, np, nullptr, st);
-  else simt_logits<float>(cp, ws, W, H, true, np, nullptr, st);
+  logits(0, logits_debug);
+  launch_fold(cp, ws, np, nq, st);
+  if (cp.rule == JD_RULE_TOPK) {   // ranks and argmax need the folded maxima; the decision writes the token
+    logits(2, nullptr);
+    launch_decide(cp, ws, st);
+    return 6;
+  }
+  launch_decide(cp, ws, st);
+  logits(1, nullptr);
   launch_locate(cp, ws, np, st);
   return 7;
 }

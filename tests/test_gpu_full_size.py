@@ -10,7 +10,7 @@ from paper_2501_19309_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 
-def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None):
+def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None, rule="sampling", top_k=1):
     """cases: list of (mode, tau or None)."""
     from paper_2501_19309_b200 import jd
     wl = I.CONFIGS[cfg]
@@ -20,13 +20,13 @@ def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None):
     rep = T.Report()
     for mode, tau in cases:
         tau = inp.tau if tau is None else tau
-        out = ver.verify(dev["H"], dev["x"], dev["dl"], tau, inp.seed, mode)
+        out = ver.verify(dev["H"], dev["x"], dev["dl"], tau, inp.seed, mode, rule=rule, top_k=top_k)
         assert ver.device_status() == jd.JD_OK
         if expect_variant:
             assert ver.launch_info()[0] == jd.VARIANTS[expect_variant]
         got = T.to_numpy(out)
-        ref = T.run_oracle(inp, mode, tau=tau, sequences=sequences)
-        T.compare(got, ref, mode, wl.M, rep)
+        ref = T.run_oracle(inp, mode, tau=tau, sequences=sequences, rule=rule, top_k=top_k)
+        T.compare(got, ref, mode, wl.M, rep, rule=rule)
     ver.close()
     del dev
     import torch
@@ -85,3 +85,14 @@ def test_cfg3_masks_independent_of_mode():
 def test_cfg4_batched_sampled_sequences():
     rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[0, 37, 63], expect_variant="batched")
     assert rep.sequences == 3
+
+
+def test_cfg1_greedy_and_top5_rules():
+    full_case(1, 0, [("standard", None), ("judge_or_standard", None)], expect_variant="fused", rule="topk", top_k=1)
+    full_case(1, 0, [("standard", None)], expect_variant="fused", rule="topk", top_k=5)
+
+
+def test_cfg4_greedy_rule_sampled_sequences():
+    rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[5, 60], expect_variant="batched",
+                       rule="topk", top_k=1)
+    assert rep.sequences == 2

@@ -13,7 +13,7 @@ MODES = ("standard", "judge", "judge_or_standard")
 
 
 def run_case(wl, data_seed, modes=MODES, variant="auto", seeds=None, tau=None, check_logits=False,
-             sequences=None, expect_variant=None):
+             sequences=None, expect_variant=None, rule="sampling", top_k=1):
     from paper_2501_19309_b200 import jd
     inp = I.make_inputs(wl, data_seed)
     dev = T.upload(inp)
@@ -23,13 +23,14 @@ def run_case(wl, data_seed, modes=MODES, variant="auto", seeds=None, tau=None, c
         for seed in (seeds or [inp.seed]):
             out = ver.alloc_outputs(wl.B, wl.M, debug_logits=check_logits)
             ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau if tau is None else tau, seed, mode,
-                       variant=variant, out=out)
+                       variant=variant, out=out, rule=rule, top_k=top_k)
             assert ver.device_status() == jd.JD_OK
             if expect_variant is not None:
                 assert ver.launch_info()[0] == jd.VARIANTS[expect_variant]
             got = T.to_numpy(out)
-            ref = T.run_oracle(inp, mode, seed=seed, tau=tau, sequences=sequences, keep_logits=check_logits)
-            T.compare(got, ref, mode, wl.M, rep)
+            ref = T.run_oracle(inp, mode, seed=seed, tau=tau, sequences=sequences, keep_logits=check_logits,
+                               rule=rule, top_k=top_k)
+            T.compare(got, ref, mode, wl.M, rep, rule=rule)
             if check_logits:
                 T.compare_logits(got["logits_debug"], ref, rep)
     ver.close()
@@ -273,4 +274,49 @@ def test_batched_matches_simt_on_every_sequence():
         assert np.mean(a["next_token"] == b["next_token"]) > 0.9      # CDF-edge cases may differ by a token
         assert np.allclose(a["row_lse"], b["row_lse"], rtol=0, atol=1e-4)
         assert np.allclose(a["p_draft"], b["p_draft"], rtol=1e-4)
+    ver.close()
+
+
+# ------------------------------------------------------------------ greedy / top-K rule (all variants)
+TOPK_CASES = [
+    ("simt", 2, 5, 100, 515, [1, 3, 515]),
+    ("simt", 3, 4, 64, 1300, [1, 40]),
+    ("fused", 1, 8, 128, 128256, [1, 5]),
+    ("fused", 4, 16, 128, 128256, [1, 2, 1000]),
+    ("fused", 2, 3, 64, 1000, [1, 1000]),
+    ("fused", 6, 15, 64, 40000 + 77, [1, 10]),        # overflow tiles + ragged last tile
+    ("batched", 8, 16, 128, 128256, [1, 4]),
+    ("batched", 3, 50, 128, 5000 + 77, [1, 100, 5077]),
+]
+
+
+@pytest.mark.parametrize("variant,B,M,d,V,ks", TOPK_CASES)
+def test_topk_rule_parity(variant, B, M, d, V, ks):
+    wl = I.CONFIGS[2].scaled("topk-%s-%d-%d-%d-%d" % (variant, B, M, d, V), B=B, M=M, d=d, V=V)
+    for k in ks:
+        rep = run_case(wl, 7, variant=variant, modes=("standard", "judge_or_standard"), seeds=[0],
+                       expect_variant=variant, rule="topk", top_k=k)
+        assert rep.sequences == 2 * B
+
+
+def test_greedy_accepts_the_targets_own_tokens_and_topk_all_accepts_everything():
+    import torch
+    wl = I.CONFIGS[1].scaled("greedy", B=3, M=6, d=128, V=30000)
+    inp = I.make_inputs(wl, 3)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    out = ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "standard", rule="topk", top_k=wl.V)
+    assert (T.to_numpy(out)["accept_len"] == wl.M).all()                 # K = V: the draft alone decides
+    # planted tokens are the target's greedy tokens here (alpha = 4): greedy verification accepts them
+    got = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "standard", rule="greedy"))
+    ref = T.run_oracle(inp, "standard", seed=0, rule="greedy")
+    T.compare(got, ref, "standard", wl.M, rule="topk")
+    assert (got["accept_len"] == ref.accept_len).all() and got["accept_len"].min() >= 1
+    # a wrong token at slot 2 is rejected and corrected to the target's token
+    x2 = dev["x"].clone()
+    x2[:, 2] = (x2[:, 2] + 1) % wl.V
+    got2 = T.to_numpy(ver.verify(dev["H"], x2, dev["dl"], 0.5, 0, "standard", rule="greedy"))
+    full = got["accept_len"] == wl.M
+    assert (got2["accept_len"][full] == 2).all()
+    assert (got2["next_token"][full] == inp.draft_tokens[full, 2]).all()
     ver.close()

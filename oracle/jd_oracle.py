@@ -31,6 +31,11 @@ greedy token argmax p_a, at a rejection as well as after a fully accepted block.
 drawn and the draft distribution plays no role. Equal logits are ordered by token id (lower id
 ranks higher), so "among the K highest" and "argmax" are unique.
 
+Final RMS normalisation (Sec. 4.1 "Model design and training": the judge reads the last embedding
+"before the RMS normalization and the LM head"): with rms_eps given, the LM head sees
+H[b,j] / sqrt(mean_k H[b,j,k]^2 + rms_eps) while the judge still reads H[b,j+1] itself. The
+normalisation gain is taken as folded into W beforehand.
+
 Readings taken where the paper is silent (all restated in the design notes):
   * the judge for draft token j reads row j+1 of H, the embedding produced by
     feeding that token (Sec. 4.1 speaks of the embedding of the current token);
@@ -123,6 +128,12 @@ def _to_f64(a: np.ndarray) -> np.ndarray:
 # --------------------------------------------------------------------------
 # the steps
 # --------------------------------------------------------------------------
+def rms_normalise(Hb: np.ndarray, eps: float) -> np.ndarray:
+    """Rows of Hb divided by sqrt(mean of squares + eps), float64 (RMSNorm without its gain)."""
+    Hd = _to_f64(Hb)
+    return Hd / np.sqrt(np.mean(Hd * Hd, axis=-1, keepdims=True) + eps)
+
+
 def project_logits(W: np.ndarray, Hb: np.ndarray, vocab_chunk: int = 8192) -> np.ndarray:
     """L[j, v] = sum_k H[j, k] * W[v, k] in float64 (Eq. 2, LM head).
 
@@ -216,7 +227,7 @@ def jd_oracle_verify(W, w_judge, b_judge: float, H, draft_tokens, draft_logits, 
                      sequences: Optional[Sequence[int]] = None, keep_logits: bool = False,
                      u_accept: Optional[np.ndarray] = None,
                      u_sample: Optional[np.ndarray] = None,
-                     rule="sampling", top_k: int = 1) -> OracleResult:
+                     rule="sampling", top_k: int = 1, rms_eps: Optional[float] = None) -> OracleResult:
     """One verification call, step by step, in float64.
 
     ``u_accept`` [B, M] / ``u_sample`` [B], when given, replace the Philox
@@ -249,7 +260,8 @@ def jd_oracle_verify(W, w_judge, b_judge: float, H, draft_tokens, draft_logits, 
 
     for b in seqs:
         Hb = _to_f64(H[b])                               # [M+1, d]
-        L = project_logits(W, H[b])                      # [M+1, V]          (Eq. 2)
+        # [M+1, V] (Eq. 2); the LM head sees the RMS-normalised rows when rms_eps is given
+        L = project_logits(W, H[b] if rms_eps is None else rms_normalise(H[b], rms_eps))
         lse_p = np.empty(M + 1)
         for j in range(M + 1):
             res.row_max[b, j], lse_p[j] = logsumexp(L[j])

@@ -71,6 +71,12 @@ typedef enum { JD_RESAMPLE_RESIDUAL = 0, JD_RESAMPLE_TARGET_P = 1 } jd_resample_
  *           only feed the q_draft output. */
 typedef enum { JD_RULE_SAMPLING = 0, JD_RULE_TOPK = 1 } jd_rule_t;
 
+/* Normalisation applied to the rows of H in front of the LM head. The paper's judge reads the last
+ * embedding "before the RMS normalization and the LM head" (Sec. 4.1): with JD_NORM_RMS the logits
+ * are W . (H[b,j] / sqrt(mean_k H[b,j,k]^2 + rms_eps)) while the judge dot product still uses
+ * H[b,j+1] as given. The norm's gain vector is expected folded into W. */
+typedef enum { JD_NORM_NONE = 0, JD_NORM_RMS = 1 } jd_norm_t;
+
 /* Kernel family used by jd_verify. AUTO picks the fastest one that supports the shape. */
 typedef enum {
   JD_VARIANT_AUTO = 0,
@@ -106,6 +112,8 @@ typedef struct {
   int32_t variant;             /* jd_variant_t; JD_VARIANT_AUTO in production */
   int32_t rule;                /* jd_rule_t */
   int32_t top_k;               /* K of JD_RULE_TOPK, >= 1; ignored by JD_RULE_SAMPLING */
+  int32_t norm;                /* jd_norm_t */
+  float rms_eps;               /* epsilon of JD_NORM_RMS, >= 0 */
   /* outputs, always written */
   int32_t* accept_len;         /* [B] number of accepted draft tokens, 0..M */
   int32_t* next_token;         /* [B] the corrected (accept_len < M) or bonus (== M) token */
@@ -183,7 +191,7 @@ jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* s
  * allocating call is made here.
  *   d, V, W, w_judge, b_judge : the head, as for jd_set_head (device pointers, 16-byte aligned)
  *   args                     : as for jd_verify (device pointers); variant must be AUTO or FUSED,
- *                              rule JD_RULE_SAMPLING, logits_debug NULL
+ *                              rule JD_RULE_SAMPLING, norm JD_NORM_NONE, logits_debug NULL
  *   device_status            : optional device pointer to one uint32 that receives the call's
  *                              device status (JD_OK, JD_ERR_TIMEOUT, JD_ERR_BAD_TOKEN); NULL to skip
  * The call uses the CURRENT device. Its first call on a device looks up the array's device

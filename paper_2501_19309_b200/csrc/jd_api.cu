@@ -112,6 +112,7 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
   w.w_sel = (float*)take(maxB * (((size_t)c.V + kVocabTile - 1) / kVocabTile * kVocabTile) * 4);
   w.p_sel = (float*)take(maxB * (size_t)c.V * 4);
   w.h_sel = (__nv_bfloat16*)take(maxB * (size_t)c.d * 2);
+  w.row_scale = (float*)take(maxR * 4);
   w.cnt = (int*)take(maxR * 4);
   w.argidx = (int*)take(maxR * 4);
   w.part_idx = (int*)take(maxR * np * 4);
@@ -139,6 +140,8 @@ jd_status_t validate(jd_handle_t h, const jd_verify_args_t* a) {
   if (a->variant < JD_VARIANT_AUTO || a->variant > JD_VARIANT_BATCHED) return JD_ERR_INVALID_ARG;
   if (a->rule != JD_RULE_SAMPLING && a->rule != JD_RULE_TOPK) return JD_ERR_INVALID_ARG;
   if (a->rule == JD_RULE_TOPK && a->top_k < 1) return JD_ERR_INVALID_ARG;
+  if (a->norm != JD_NORM_NONE && a->norm != JD_NORM_RMS) return JD_ERR_INVALID_ARG;
+  if (a->norm == JD_NORM_RMS && !(a->rms_eps >= 0.f)) return JD_ERR_INVALID_ARG;
   return JD_OK;
 }
 
@@ -251,6 +254,7 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   cp.tau = a->tau; cp.b_judge = h->b_judge; cp.seed = a->seed;
   cp.mode = a->mode; cp.resample = a->resample;
   cp.rule = a->rule; cp.top_k = a->top_k;
+  cp.norm = a->norm; cp.rms_eps = a->rms_eps;
   cp.accept_len = a->accept_len; cp.next_token = a->next_token;
   cp.judge_scores = a->judge_scores; cp.p_draft = a->p_draft;
   cp.q_draft = a->q_draft; cp.masks = a->masks;
@@ -278,8 +282,12 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
       return JD_ERR_CUDA;
   }
   int launches = 0;
+  if (a->norm == JD_NORM_RMS) {   // per-row normalisation factors, read by every variant
+    launch_row_scale(cp, h->ws, a->H, c.dtype, st);
+    launches = 1;
+  }
   if (variant == JD_VARIANT_SIMT) {
-    launches = run_simt(cp, h->ws, h->W, h->w_judge, a->H, c.dtype, a->logits_debug, st);
+    launches += run_simt(cp, h->ws, h->W, h->w_judge, a->H, c.dtype, a->logits_debug, st);
   } else if (variant == JD_VARIANT_BATCHED) {
     FusedPlan plan2;   // second pass: B rows through the fused kernel
     if (!fused_supported(c.dtype, a->B, c.d, c.V, h->num_sms, &plan2)) return JD_ERR_UNSUPPORTED;
@@ -288,14 +296,16 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
         !make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)a->B, (uint64_t)c.d, (uint32_t)plan2.n_pad))
       return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
-    launches = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, a->H, h->w_judge, h->num_sms, st, h->side, &err);
-    if (launches < 0) return JD_ERR_CUDA;
+    const int n = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, a->H, h->w_judge, h->num_sms, st, h->side, &err);
+    if (n < 0) return JD_ERR_CUDA;
+    launches += n;
   } else {
     CUtensorMap tm_h;
     if (!make_tensor_map(&tm_h, a->H, (uint64_t)R, (uint64_t)c.d, (uint32_t)plan.n_pad)) return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
-    launches = run_fused(cp, h->ws, h->tm_w, tm_h, a->H, h->w_judge, plan, st, &err);
-    if (launches < 0) return JD_ERR_CUDA;
+    const int n = run_fused(cp, h->ws, h->tm_w, tm_h, a->H, h->w_judge, plan, st, &err);
+    if (n < 0) return JD_ERR_CUDA;
+    launches += n;
   }
   if (cudaGetLastError() != cudaSuccess) return JD_ERR_CUDA;
   h->last_stream = st;

@@ -160,6 +160,7 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       bool have_g = false;
       int above = 0, cand = 0x7F7F7F7F;
       float g_ref = 0.f, rmax = 0.f;
+      const float sc = (cp.norm == JD_NORM_RMS && row < R) ? ws.row_scale[row] : 1.f;
       if (kCount && row < R) {
         rmax = ws.row_max[row];
         if (x >= 0) g_ref = ws.gath[row];
@@ -168,6 +169,8 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       for (int c0 = 0; c0 < kTileN; c0 += 32) {
         float v[32];
         tmem_ld32(lane_base + (uint32_t)(buf * kTileN + c0), v);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) v[k] *= sc;
         const int nvalid = cp.V - (v0 + c0);   // columns of this chunk that exist (>= 32 except at the tail)
         if (nvalid < 32) {
 #pragma unroll

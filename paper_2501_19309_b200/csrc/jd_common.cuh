@@ -38,6 +38,7 @@ struct Workspace {
   float* w_sel;        // [maxB][V]  sampling weights (SIMT variant); in the batched variant the selected
                        //            draft rows, tile-major [ceil(V/128)][B][128]
   float* p_sel;        // [maxB][V]  p of the selected row (same)
+  float* row_scale;    // [maxR] 1 / sqrt(mean square + eps) of every row of H (JD_NORM_RMS)
   int* cnt;            // [maxR] top-K rule: entries of the row that rank above the drafted token
   int* argidx;         // [maxR] top-K rule: lowest token id that attains the row maximum
   int* part_idx;       // [maxR][np] top-K rule, fused variant: per-CTA argmax candidates
@@ -121,6 +122,8 @@ struct CallParams {
   uint64_t seed;
   int mode, resample;
   int rule, top_k;
+  int norm;
+  float rms_eps;
   int32_t* accept_len;
   int32_t* next_token;
   float* judge_scores;

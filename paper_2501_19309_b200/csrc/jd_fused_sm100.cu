@@ -71,6 +71,7 @@ struct Misc {
   float lse[N_PAD];         // log-normaliser of every row
   float qlse[N_PAD];
   int x_row[N_PAD];         // drafted token of row r (rows j < M), -1 otherwise
+  float scale[N_PAD];       // normalisation factor of the row in TMEM column r (1 without JD_NORM_RMS)
   int glist[N_PAD];
   // per sequence (B <= N_PAD / 2 in the full mode, B <= N_PAD in sample-only mode)
   int sel_row[N_PAD];
@@ -94,7 +95,7 @@ struct Misc {
 // or from the overflow copy in shared memory
 template <int N_PAD>
 __device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, int ts, uint32_t tmem_lane_base,
-                                            const float* ovf, int tid, float* v0, float* v1) {
+                                            const float* ovf, int tid, const float* sc, float* v0, float* v1) {
   uint32_t a[16], b[16];
 #pragma unroll
   for (int k = 0; k < 16; ++k) { a[k] = 0u; b[k] = 0u; }
@@ -114,12 +115,16 @@ __device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, in
   }
   tmem_wait_ld32(a, b);
 #pragma unroll
-  for (int k = 0; k < 16; ++k) { v0[k] = __uint_as_float(a[k]); v1[k] = __uint_as_float(b[k]); }
+  for (int k = 0; k < 16; ++k) {
+    const float f = sc[c0 + k];   // row normalisation factor (shared memory)
+    v0[k] = __uint_as_float(a[k]) * f;
+    v1[k] = __uint_as_float(b[k]) * f;
+  }
 }
 // logits of row r in tiles i0 .. i0+7 (those below T) for this thread's lane, fetched together
 template <int N_PAD>
 __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, int ts, uint32_t tmem_lane_base,
-                                           const float* ovf, int tid, float* out) {
+                                           const float* ovf, int tid, float f, float* out) {
   uint32_t raw[8];
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
@@ -132,7 +137,7 @@ __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, int 
   }
   tmem_wait_ld8(raw);
 #pragma unroll
-  for (int u = 0; u < 8; ++u) out[u] = __uint_as_float(raw[u]);
+  for (int u = 0; u < 8; ++u) out[u] = __uint_as_float(raw[u]) * f;
 }
 
 // Reduces 16 per-lane values over the 32 lanes of a warp with 16 shuffles instead of 80: every
@@ -217,6 +222,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
     }
     ms.x_row[tid] = x;
+    float f = 1.f;   // normalisation factor of the row held in TMEM column tid
+    if (cp.norm == JD_NORM_RMS && tid < R) f = ws.row_scale[fp.sample_only ? ws.sel_row[tid] : tid];
+    ms.scale[tid] = f;
   }
   if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ms.tmem_base)),
@@ -410,7 +418,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int r = ms.glist[e], x = ms.x_row[r];
         const int i = x / kVocabTile - t0;
         float one[8];
-        load_cols8<N_PAD>(i, i + 1, r, n_ovf, ts, tmem_lane_base, ovf, tid, one);
+        load_cols8<N_PAD>(i, i + 1, r, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[r], one);
         if (tid == (x % kVocabTile)) ws.gath[r] = one[0];
       }
     }
@@ -422,7 +430,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (ok) {
         for (int i0 = 0; i0 < T; i0 += 2) {
           float v0[16], v1[16];
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, v0, v1);
           const bool val0 = (t0 + i0) * kVocabTile + tid < V;
           const bool val1 = (i0 + 1 < T) && ((t0 + i0 + 1) * kVocabTile + tid < V);
           if (val0) {
@@ -451,7 +459,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (ok) {
         for (int i0 = 0; i0 < T; i0 += 2) {
           float v0[16], v1[16];
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, v0, v1);
           const bool val0 = (t0 + i0) * kVocabTile + tid < V;
           const bool val1 = (i0 + 1 < T) && ((t0 + i0 + 1) * kVocabTile + tid < V);
           if (val0) {
@@ -507,7 +515,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
         for (int i0 = 0; i0 < T; i0 += 2) {
           float v0[16], v1[16];
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, v0, v1);
           const int vg0 = (t0 + i0) * kVocabTile + tid, vg1 = vg0 + kVocabTile;
           const bool val0 = vg0 < V, val1 = (i0 + 1 < T) && vg1 < V;
 #pragma unroll
@@ -684,7 +692,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             d0[k] = __ldg(base0 + kk * kVocabTile);
             d1[k] = __ldg(base1 + kk * kVocabTile);
           }
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, v0, v1);
 #pragma unroll
           for (int k = 0; k < 16; ++k) {
             const float p0 = fast_exp2(fmaf(v0[k], kLog2e, -lp2[k])), q0 = fast_exp2(fmaf(d0[k], kLog2e, -lq2[k]));
@@ -729,7 +737,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           for (int q = 0; q < 4; ++q) {
             const int b = min(b0 + q, cp.B - 1);
             const int col = fp.sample_only ? b : ms.sel_row[b];   // TMEM column of this sequence's selected row
-            load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, lg[q]);
+            load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], lg[q]);
           }
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -867,7 +875,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                                               : dlrow + vg;
             dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(src) : 0.f;
           }
-          load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, lg);
+          load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], lg);
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int vg = (t0 + i0 + u) * kVocabTile + tid;

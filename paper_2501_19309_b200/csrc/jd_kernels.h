@@ -12,6 +12,7 @@ int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const voi
              float* logits_debug, cudaStream_t st);
 int launch_q_stats(const CallParams& cp, const Workspace& ws, cudaStream_t st);   // returns partials per draft row
 void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, const void* w, int dtype, cudaStream_t st);
+void launch_row_scale(const CallParams& cp, const Workspace& ws, const void* H, int dtype, cudaStream_t st);
 void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st);
 void launch_decide(const CallParams& cp, const Workspace& ws, cudaStream_t st);
 void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream_t st);

@@ -29,6 +29,7 @@ __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, 
   __shared__ float s_m[4][kSimtRows], s_s[4][kSimtRows];
   __shared__ double s_d[2][4][kSimtRows];
   __shared__ int s_row[kSimtRows];
+  __shared__ float s_scale[kSimtRows];
 
   constexpr bool kSample = (kMode == 1);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -40,6 +41,7 @@ __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, 
   if (tid < kSimtRows) {
     const int r = r0 + tid;
     s_row[tid] = (r < R) ? (kSample ? ws.sel_row[r] : r) : -1;
+    s_scale[tid] = (cp.norm == JD_NORM_RMS && s_row[tid] >= 0) ? ws.row_scale[s_row[tid]] : 1.f;
   }
   __syncthreads();
 
@@ -74,6 +76,9 @@ __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, 
     }
     __syncthreads();
   }
+
+#pragma unroll
+  for (int i = 0; i < kSimtRows; ++i) acc[i] *= s_scale[i];   // 1 when no normalisation is asked for
 
   const bool valid_v = v < V;
   if (kMode == 2) {
@@ -194,6 +199,25 @@ __global__ void __launch_bounds__(256) q_stats_kernel(CallParams cp, Workspace w
       if (x < 0 || x >= V) { set_status(ws.status, JD_ERR_BAD_TOKEN); x = min(max(x, 0), V - 1); }
       ws.qgath[bm] = row[x];
     }
+  }
+}
+
+// Row normalisation factors of JD_NORM_RMS: one block per row, 1 / sqrt(mean_k H[row,k]^2 + eps).
+template <typename T>
+__global__ void __launch_bounds__(256) row_scale_kernel(CallParams cp, Workspace ws, const T* __restrict__ H) {
+  __shared__ float s_p[8];
+  const int row = blockIdx.x;
+  const T* h = H + (size_t)row * cp.d;
+  float acc = 0.f;
+  for (int k = threadIdx.x; k < cp.d; k += blockDim.x) { const float x = to_float<T>(h[k]); acc = fmaf(x, x, acc); }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) s_p[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < 8; ++i) t += s_p[i];
+    ws.row_scale[row] = rsqrtf(t / (float)cp.d + cp.rms_eps);
   }
 }
 
@@ -341,6 +365,12 @@ void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, cons
     judge_dot_kernel<__nv_bfloat16><<<cp.B * cp.M, 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H, (const __nv_bfloat16*)w);
   else
     judge_dot_kernel<float><<<cp.B * cp.M, 256, 0, st>>>(cp, ws, (const float*)H, (const float*)w);
+}
+
+void launch_row_scale(const CallParams& cp, const Workspace& ws, const void* H, int dtype, cudaStream_t st) {
+  const int R = cp.B * (cp.M + 1);
+  if (dtype == JD_DTYPE_BF16) row_scale_kernel<__nv_bfloat16><<<R, 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H);
+  else row_scale_kernel<float><<<R, 256, 0, st>>>(cp, ws, (const float*)H);
 }
 
 void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st) {

@@ -76,6 +76,7 @@ extern "C" jd_status_t jd_verify_static(int32_t d, int32_t V, const void* W, con
   if (a->resample < JD_RESAMPLE_RESIDUAL || a->resample > JD_RESAMPLE_TARGET_P) return JD_ERR_INVALID_ARG;
   if (a->variant != JD_VARIANT_AUTO && a->variant != JD_VARIANT_FUSED) return JD_ERR_INVALID_ARG;
   if (a->rule != JD_RULE_SAMPLING) return JD_ERR_UNSUPPORTED;   // the fixed scratch has no rank counters
+  if (a->norm != JD_NORM_NONE) return JD_ERR_UNSUPPORTED;       // nor row normalisation factors
   if (!aligned16(W) || !aligned16(w_judge) || !aligned16(a->H)) return JD_ERR_INVALID_ARG;
   // the fixed scratch holds at most 96 rows: larger blocks are refused, never truncated
   if ((int64_t)a->B * (a->M + 1) > kStaticMaxRows) return JD_ERR_UNSUPPORTED;
@@ -134,6 +135,7 @@ extern "C" jd_status_t jd_verify_static(int32_t d, int32_t V, const void* W, con
   cp.tau = a->tau; cp.b_judge = b_judge; cp.seed = a->seed;
   cp.mode = a->mode; cp.resample = a->resample;
   cp.rule = JD_RULE_SAMPLING; cp.top_k = 1;
+  cp.norm = JD_NORM_NONE; cp.rms_eps = 0.f;
   cp.accept_len = a->accept_len; cp.next_token = a->next_token;
   cp.judge_scores = a->judge_scores; cp.p_draft = a->p_draft;
   cp.q_draft = a->q_draft; cp.masks = a->masks;

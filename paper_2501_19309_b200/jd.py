@@ -24,6 +24,7 @@ JD_MODE_STANDARD, JD_MODE_JUDGE, JD_MODE_JUDGE_OR_STANDARD = 0, 1, 2
 JD_RESAMPLE_RESIDUAL, JD_RESAMPLE_TARGET_P = 0, 1
 JD_VARIANT_AUTO, JD_VARIANT_SIMT, JD_VARIANT_FUSED, JD_VARIANT_BATCHED = 0, 1, 2, 3
 JD_RULE_SAMPLING, JD_RULE_TOPK = 0, 1
+JD_NORM_NONE, JD_NORM_RMS = 0, 1
 
 MODES = {"standard": JD_MODE_STANDARD, "judge": JD_MODE_JUDGE, "judge_or_standard": JD_MODE_JUDGE_OR_STANDARD}
 RESAMPLE = {"residual": JD_RESAMPLE_RESIDUAL, "target_p": JD_RESAMPLE_TARGET_P}
@@ -43,7 +44,7 @@ class jd_config_t(C.Structure):
 class jd_verify_args_t(C.Structure):
     _fields_ = [("B", C.c_int32), ("M", C.c_int32), ("H", C.c_void_p), ("draft_tokens", C.c_void_p),
                 ("draft_logits", C.c_void_p), ("tau", C.c_float), ("seed", C.c_uint64), ("mode", C.c_int32),
-                ("resample", C.c_int32), ("variant", C.c_int32), ("rule", C.c_int32), ("top_k", C.c_int32),
+                ("resample", C.c_int32), ("variant", C.c_int32), ("rule", C.c_int32), ("top_k", C.c_int32), ("norm", C.c_int32), ("rms_eps", C.c_float),
                 ("accept_len", C.c_void_p), ("next_token", C.c_void_p), ("judge_scores", C.c_void_p),
                 ("p_draft", C.c_void_p), ("q_draft", C.c_void_p), ("masks", C.c_void_p),
                 ("row_max", C.c_void_p), ("row_lse", C.c_void_p), ("logits_debug", C.c_void_p)]
@@ -210,7 +211,7 @@ class Verifier:
 
     def make_args(self, H, draft_tokens, draft_logits, tau: float, seed: int, mode="judge_or_standard",
                   resample="residual", variant="auto", out: Optional[dict] = None, host: bool = False,
-                  rule="sampling", top_k: int = 1):
+                  rule="sampling", top_k: int = 1, rms_eps: Optional[float] = None):
         B, Mp1, _ = H.shape
         M = Mp1 - 1
         if out is None:
@@ -224,13 +225,15 @@ class Verifier:
         a.variant = VARIANTS[variant] if isinstance(variant, str) else int(variant)
         a.rule = RULES[rule] if isinstance(rule, str) else int(rule)
         a.top_k = 1 if rule == "greedy" else int(top_k)
+        a.norm = JD_NORM_NONE if rms_eps is None else JD_NORM_RMS
+        a.rms_eps = 0.0 if rms_eps is None else float(rms_eps)
         for k in OUTPUT_NAMES:
             setattr(a, k, out[k].data_ptr() if out.get(k) is not None else None)
         return a, out
 
     def verify(self, H, draft_tokens, draft_logits, tau: float, seed: int, mode="judge_or_standard",
                resample="residual", variant="auto", out: Optional[dict] = None, stream=None,
-               rule="sampling", top_k: int = 1) -> dict:
+               rule="sampling", top_k: int = 1, rms_eps: Optional[float] = None) -> dict:
         """Enqueues one verification on ``stream`` (default: torch's current stream); returns the
         dict of output tensors (device)."""
         t = self.torch
@@ -238,7 +241,7 @@ class Verifier:
         assert draft_tokens.dtype == t.int32 and draft_tokens.is_contiguous() and draft_tokens.is_cuda
         assert draft_logits.dtype == t.float32 and draft_logits.is_contiguous() and draft_logits.is_cuda
         a, out = self.make_args(H, draft_tokens, draft_logits, tau, seed, mode, resample, variant, out,
-                                rule=rule, top_k=top_k)
+                                rule=rule, top_k=top_k, rms_eps=rms_eps)
         s = stream if stream is not None else t.cuda.current_stream(self.device)
         st = jd_verify(self.h, a, s.cuda_stream)
         if st != JD_OK:

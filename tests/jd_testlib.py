@@ -60,10 +60,11 @@ def to_numpy(out: dict) -> dict:
 
 
 def run_oracle(inp: I.Inputs, mode, seed=None, tau=None, resample="residual", sequences=None, keep_logits=False,
-               rule="sampling", top_k=1):
+               rule="sampling", top_k=1, rms_eps=None):
     return O.jd_oracle_verify(inp.W, inp.w_judge, inp.b_judge, inp.H, inp.draft_tokens, inp.draft_logits,
                               inp.tau if tau is None else tau, inp.seed if seed is None else seed,
-                              mode, resample, sequences=sequences, keep_logits=keep_logits, rule=rule, top_k=top_k)
+                              mode, resample, sequences=sequences, keep_logits=keep_logits, rule=rule, top_k=top_k,
+                              rms_eps=rms_eps)
 
 
 @dataclasses.dataclass

@@ -13,7 +13,7 @@ MODES = ("standard", "judge", "judge_or_standard")
 
 
 def run_case(wl, data_seed, modes=MODES, variant="auto", seeds=None, tau=None, check_logits=False,
-             sequences=None, expect_variant=None, rule="sampling", top_k=1):
+             sequences=None, expect_variant=None, rule="sampling", top_k=1, rms_eps=None):
     from paper_2501_19309_b200 import jd
     inp = I.make_inputs(wl, data_seed)
     dev = T.upload(inp)
@@ -23,13 +23,13 @@ def run_case(wl, data_seed, modes=MODES, variant="auto", seeds=None, tau=None, c
         for seed in (seeds or [inp.seed]):
             out = ver.alloc_outputs(wl.B, wl.M, debug_logits=check_logits)
             ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau if tau is None else tau, seed, mode,
-                       variant=variant, out=out, rule=rule, top_k=top_k)
+                       variant=variant, out=out, rule=rule, top_k=top_k, rms_eps=rms_eps)
             assert ver.device_status() == jd.JD_OK
             if expect_variant is not None:
                 assert ver.launch_info()[0] == jd.VARIANTS[expect_variant]
             got = T.to_numpy(out)
             ref = T.run_oracle(inp, mode, seed=seed, tau=tau, sequences=sequences, keep_logits=check_logits,
-                               rule=rule, top_k=top_k)
+                               rule=rule, top_k=top_k, rms_eps=rms_eps)
             T.compare(got, ref, mode, wl.M, rep, rule=rule)
             if check_logits:
                 T.compare_logits(got["logits_debug"], ref, rep)
@@ -319,4 +319,43 @@ def test_greedy_accepts_the_targets_own_tokens_and_topk_all_accepts_everything()
     full = got["accept_len"] == wl.M
     assert (got2["accept_len"][full] == 2).all()
     assert (got2["next_token"][full] == inp.draft_tokens[full, 2]).all()
+    ver.close()
+
+
+# ------------------------------------------------------------------ final RMS normalisation (all variants)
+NORM_CASES = [
+    ("simt", 2, 5, 100, 515, "f32"),
+    ("simt", 3, 4, 192, 1300, "bf16"),
+    ("fused", 1, 8, 256, 128256, "bf16"),
+    ("fused", 4, 16, 128, 40000 + 77, "bf16"),
+    ("fused", 6, 15, 64, 128256, "bf16"),            # overflow tiles
+    ("batched", 8, 16, 128, 128256, "bf16"),
+    ("batched", 40, 2, 128, 33000, "bf16"),
+]
+
+
+@pytest.mark.parametrize("variant,B,M,d,V,dtype", NORM_CASES)
+def test_rms_normalised_head_parity(variant, B, M, d, V, dtype):
+    wl = I.CONFIGS[2].scaled("norm-%s-%d-%d-%d-%d" % (variant, B, M, d, V), B=B, M=M, d=d, V=V, dtype=dtype,
+                             alpha_range=(2.0, 9.0))           # rows of clearly different norms
+    seqs = None if B <= 8 else [0, B // 2, B - 1]
+    rep = run_case(wl, 11, variant=variant, modes=("judge_or_standard", "standard"), seeds=[0, 1],
+                   sequences=seqs, expect_variant=variant, rms_eps=1e-5, check_logits=(variant == "simt"))
+    assert rep.sequences == 4 * (B if seqs is None else len(seqs))
+    if variant == "fused":
+        rep = run_case(wl, 11, variant=variant, modes=("standard",), seeds=[0], rule="greedy", rms_eps=1e-5)
+
+
+def test_rms_norm_makes_target_side_scale_invariant_on_device():
+    import torch
+    wl = I.CONFIGS[1].scaled("inv", B=2, M=6, d=256, V=20000)
+    inp = I.make_inputs(wl, 2)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    a = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 4, "standard", rms_eps=0.0))
+    H4 = (dev["H"].float() * 4.0).to(torch.bfloat16)            # exact in bf16: a power of two
+    b = T.to_numpy(ver.verify(H4, dev["x"], dev["dl"], 0.5, 4, "standard", rms_eps=0.0))
+    assert np.allclose(a["row_lse"], b["row_lse"], rtol=0, atol=1e-4)
+    assert np.array_equal(a["accept_len"], b["accept_len"]) and np.array_equal(a["masks"] & 1, b["masks"] & 1)
+    assert not np.allclose(a["judge_scores"], b["judge_scores"])     # the judge reads the raw rows
     ver.close()

@@ -36,6 +36,14 @@ Final RMS normalisation (Sec. 4.1 "Model design and training": the judge reads t
 H[b,j] / sqrt(mean_k H[b,j,k]^2 + rms_eps) while the judge still reads H[b,j+1] itself. The
 normalisation gain is taken as folded into W beforehand.
 
+8-bit head (the paper runs its targets with 8-bit weights, Table 1 caption and App. B.3): with
+w_scale given, W holds FP8 E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no
+infinities) and the logical weight is w_scale[v] * e4m3(W[v,k]). The rows of H are then quantised
+the same way before the LM head: s_r = max_k |H[r,k]| / 448 and h8 = e4m3(round-to-nearest-even,
+saturating, of H[r,k] * (448 / max_k |H[r,k]|)), the scale and the product in float32 as the
+kernel takes them, so that both sides pick the same codes. The logit is
+w_scale[v] * s_r * sum_k e4m3(W[v,k]) * h8[r,k]; the judge still reads the unquantised row.
+
 Readings taken where the paper is silent (all restated in the design notes):
   * the judge for draft token j reads row j+1 of H, the embedding produced by
     feeding that token (Sec. 4.1 speaks of the embedding of the current token);
@@ -128,6 +136,44 @@ def _to_f64(a: np.ndarray) -> np.ndarray:
 # --------------------------------------------------------------------------
 # the steps
 # --------------------------------------------------------------------------
+# --------------------------------------------------------------------------
+# FP8 E4M3 ("fn": finite, no infinities; 0x7F / 0xFF are NaN), from the format's definition
+# --------------------------------------------------------------------------
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    """float64 values of E4M3 codes (uint8): (-1)^s 2^(e-7) (1 + m/8), e = 0: (-1)^s 2^-6 m/8."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    sgn = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = (c & 0x7).astype(np.float64)
+    val = np.where(e == 0, np.ldexp(m / 8.0, -6), np.ldexp(1.0 + m / 8.0, e - 7))
+    val = np.where((c & 0x7F) == 0x7F, np.nan, val)
+    return sgn * val
+
+
+def e4m3_round(x: np.ndarray) -> np.ndarray:
+    """Nearest E4M3 value of every float32 in x, ties to even, saturating at +-448; float64."""
+    x = np.asarray(x, dtype=np.float32).astype(np.float64)
+    a = np.minimum(np.abs(x), 448.0)
+    # spacing of the E4M3 grid around a: 2^(floor(log2 a) - 3), but never finer than 2^-9
+    ex = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))
+    q = np.ldexp(1.0, (ex - 3).astype(np.int64))
+    r = np.round(a / q) * q                   # numpy rounds halves to even; a / q is exact
+    return np.copysign(np.minimum(r, 448.0), x)
+
+
+def quantise_rows_e4m3(Hb: np.ndarray) -> tuple:
+    """Per-row E4M3 quantisation in the kernel's arithmetic: returns (values [rows, d] float64 on
+    the E4M3 grid, scale [rows] float64) with H ~ scale * values."""
+    Hf = _to_f64(Hb).astype(np.float32)                    # bf16 / f32 inputs are exact in float32
+    amax = np.max(np.abs(Hf), axis=-1, keepdims=True).astype(np.float32)
+    safe = np.where(amax > 0, amax, np.float32(1.0)).astype(np.float32)
+    inv = (np.float32(448.0) / safe).astype(np.float32)    # float32 division, round to nearest
+    scaled = (Hf * inv).astype(np.float32)                 # float32 product, round to nearest
+    vals = e4m3_round(scaled)
+    scale = (amax / np.float32(448.0)).astype(np.float32)  # float32 division
+    return vals, scale[..., 0].astype(np.float64)
+
+
 def rms_normalise(Hb: np.ndarray, eps: float) -> np.ndarray:
     """Rows of Hb divided by sqrt(mean of squares + eps), float64 (RMSNorm without its gain)."""
     Hd = _to_f64(Hb)
@@ -227,7 +273,8 @@ def jd_oracle_verify(W, w_judge, b_judge: float, H, draft_tokens, draft_logits, 
                      sequences: Optional[Sequence[int]] = None, keep_logits: bool = False,
                      u_accept: Optional[np.ndarray] = None,
                      u_sample: Optional[np.ndarray] = None,
-                     rule="sampling", top_k: int = 1, rms_eps: Optional[float] = None) -> OracleResult:
+                     rule="sampling", top_k: int = 1, rms_eps: Optional[float] = None,
+                     w_scale: Optional[np.ndarray] = None) -> OracleResult:
     """One verification call, step by step, in float64.
 
     ``u_accept`` [B, M] / ``u_sample`` [B], when given, replace the Philox
@@ -261,7 +308,19 @@ def jd_oracle_verify(W, w_judge, b_judge: float, H, draft_tokens, draft_logits, 
     for b in seqs:
         Hb = _to_f64(H[b])                               # [M+1, d]
         # [M+1, V] (Eq. 2); the LM head sees the RMS-normalised rows when rms_eps is given
-        L = project_logits(W, H[b] if rms_eps is None else rms_normalise(H[b], rms_eps))
+        if w_scale is None:
+            L = project_logits(W, H[b] if rms_eps is None else rms_normalise(H[b], rms_eps))
+        else:
+            # 8-bit head: E4M3 weights with per-row scales, rows of H quantised per row
+            h8, s_h = quantise_rows_e4m3(H[b])
+            L = np.empty((M + 1, V), dtype=np.float64)
+            for v0 in range(0, V, 8192):
+                v1 = min(V, v0 + 8192)
+                L[:, v0:v1] = h8 @ e4m3_decode(W[v0:v1]).T
+            L *= np.asarray(w_scale, dtype=np.float64)[None, :] * s_h[:, None]
+            if rms_eps is not None:
+                Hd = _to_f64(H[b])
+                L /= np.sqrt(np.mean(Hd * Hd, axis=-1, keepdims=True) + rms_eps)
         lse_p = np.empty(M + 1)
         for j in range(M + 1):
             res.row_max[b, j], lse_p[j] = logsumexp(L[j])

@@ -48,7 +48,10 @@ typedef enum {
   JD_ERR_BAD_TOKEN = 7    /* device status: a draft token was outside [0, V) and was clamped */
 } jd_status_t;
 
-typedef enum { JD_DTYPE_F32 = 0, JD_DTYPE_BF16 = 1 } jd_dtype_t;
+/* Storage type of the head. F32 / BF16: W, H and w_judge all have that type. FP8_E4M3: W holds
+ * FP8 E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities) with one
+ * float32 scale per vocabulary row, registered with jd_set_head_fp8; H and w_judge are bf16. */
+typedef enum { JD_DTYPE_F32 = 0, JD_DTYPE_BF16 = 1, JD_DTYPE_FP8_E4M3 = 2 } jd_dtype_t;
 
 /* Which tests form the accept mask (Sec. 4.1 "Inference"): the standard test alone (Eq. 4),
  * the judge alone, or their logical OR (the paper's judge decoding). */
@@ -102,7 +105,8 @@ typedef struct jd_handle_s* jd_handle_t;
 typedef struct {
   int32_t B;                   /* sequences in this call, 1..max_B */
   int32_t M;                   /* draft tokens per sequence, 1..max_M */
-  const void* H;               /* [B, M+1, d] embeddings, dtype of the handle, 16-byte aligned */
+  const void* H;               /* [B, M+1, d] embeddings, dtype of the handle (bf16 for an FP8 head),
+                                  16-byte aligned */
   const int32_t* draft_tokens; /* [B, M] drafted token ids x_j in [0, V) */
   const float* draft_logits;   /* [B, M, V] draft-model logits; q_j = softmax at temperature 1 */
   float tau;                   /* judge threshold in [0, 1]; accept iff score > tau (strict) */
@@ -150,6 +154,17 @@ jd_status_t jd_destroy(jd_handle_t h);
  * The judge head is the paper's linear map R^d -> R (Sec. 4.1 "Model design and training",
  * App. B.1). Builds the TMA descriptors of W. Must precede jd_verify. */
 jd_status_t jd_set_head(jd_handle_t h, const void* W, const void* w_judge, float b_judge);
+
+/* 8-bit head (the paper runs its targets with 8-bit weights: Table 1 caption, App. B.3). Handles
+ * created with JD_DTYPE_FP8_E4M3 register W8 [V, d] (uint8 E4M3 codes, 16-byte aligned) and w_scale [V]
+ * (float32): the logical weight is w_scale[v] * e4m3(W8[v,k]). Every call then quantises the rows
+ * of H the same way on the device, s_r = max_k |H[r,k]| / 448 and h8 = e4m3(H[r,k] * 448 / max_k |H[r,k]|)
+ * rounded to nearest even, and the tensor cores multiply FP8 by FP8 with fp32 accumulation:
+ * L[r,v] = w_scale[v] * s_r * sum_k e4m3(W8[v,k]) * h8[r,k]. The judge still reads the bf16 rows.
+ * w_judge [d] is bf16. Pointers are borrowed like those of jd_set_head. Requires d % 128 == 0 for
+ * the tensor-core variant (the CUDA-core variant takes any d); the batched variant has no FP8 form. */
+jd_status_t jd_set_head_fp8(jd_handle_t h, const void* W8, const float* w_scale, const void* w_judge,
+                            float b_judge);
 
 /* One verification call (steps 1-5 above) enqueued on `cuda_stream` (a cudaStream_t, NULL =
  * default stream). Host-side checks return JD_ERR_INVALID_ARG / JD_ERR_UNSUPPORTED before

@@ -19,6 +19,7 @@ struct jd_handle_s {
   Workspace ws;
   const void* W;
   const void* w_judge;
+  const float* w_scale;    // FP8 head: one scale per vocabulary row
   float b_judge;
   bool head_set;
   bool tm_w_ok;
@@ -58,14 +59,16 @@ EncodeTiledFn encode_tiled_fn() {
 
 // bf16 [rows, d] row-major tensor, box = 64 columns (128 bytes) x box_rows, 128-byte swizzle,
 // out-of-range rows read as zero.
-bool make_tensor_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t d, uint32_t box_rows) {
+bool make_tensor_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t d, uint32_t box_rows,
+                     bool bytes = false) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
+  // bf16: 64 elements per box row; 8-bit codes: 128 elements; 128 bytes either way
   const cuuint64_t dims[2] = {d, rows};
-  const cuuint64_t strides[1] = {d * 2};
-  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint64_t strides[1] = {bytes ? d : d * 2};
+  const cuuint32_t box[2] = {bytes ? 128u : 64u, box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(tm, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -75,7 +78,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 bool config_ok(const jd_config_t* c) {
   if (!c) return false;
   if (c->max_B < 1 || c->max_M < 1 || c->d < 1 || c->V < 2) return false;
-  if (c->dtype != JD_DTYPE_F32 && c->dtype != JD_DTYPE_BF16) return false;
+  if (c->dtype != JD_DTYPE_F32 && c->dtype != JD_DTYPE_BF16 && c->dtype != JD_DTYPE_FP8_E4M3) return false;
   if ((int64_t)c->max_B * (c->max_M + 1) > (1 << 20)) return false;
   return true;
 }
@@ -112,6 +115,8 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
   w.w_sel = (float*)take(maxB * (((size_t)c.V + kVocabTile - 1) / kVocabTile * kVocabTile) * 4);
   w.p_sel = (float*)take(maxB * (size_t)c.V * 4);
   w.h_sel = (__nv_bfloat16*)take(maxB * (size_t)c.d * 2);
+  w.h8 = (uint8_t*)take(c.dtype == JD_DTYPE_FP8_E4M3 ? maxR * (size_t)c.d : 16);
+  w.h_scale = (float*)take(maxR * 4);
   w.row_scale = (float*)take(maxR * 4);
   w.cnt = (int*)take(maxR * 4);
   w.argidx = (int*)take(maxR * 4);
@@ -124,7 +129,8 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
   return off;
 }
 
-size_t elem_size(int dtype) { return dtype == JD_DTYPE_BF16 ? 2 : 4; }
+// bytes per element of H and w_judge (an FP8 head keeps bf16 activations)
+size_t elem_size(int dtype) { return dtype == JD_DTYPE_F32 ? 4 : 2; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -225,8 +231,24 @@ jd_status_t jd_destroy(jd_handle_t h) {
   return JD_OK;
 }
 
+jd_status_t jd_set_head_fp8(jd_handle_t h, const void* W8, const float* w_scale, const void* w_judge, float b_judge) {
+  if (!h || !W8 || !w_scale || !w_judge) return JD_ERR_INVALID_ARG;
+  if (h->cfg.dtype != JD_DTYPE_FP8_E4M3) return JD_ERR_INVALID_ARG;
+  if (!aligned16(W8) || !aligned16(w_judge)) return JD_ERR_INVALID_ARG;
+  h->W = W8;
+  h->w_scale = w_scale;
+  h->w_judge = w_judge;
+  h->b_judge = b_judge;
+  h->head_set = true;
+  h->tm_w_ok = false;
+  if (h->cfg.d % 128 == 0)
+    h->tm_w_ok = make_tensor_map(&h->tm_w, W8, (uint64_t)h->cfg.V, (uint64_t)h->cfg.d, 128, true);
+  return JD_OK;
+}
+
 jd_status_t jd_set_head(jd_handle_t h, const void* W, const void* w_judge, float b_judge) {
   if (!h || !W || !w_judge) return JD_ERR_INVALID_ARG;
+  if (h->cfg.dtype == JD_DTYPE_FP8_E4M3) return JD_ERR_INVALID_ARG;   // use jd_set_head_fp8
   if (!aligned16(W) || !aligned16(w_judge)) return JD_ERR_INVALID_ARG;
   h->W = W;
   h->w_judge = w_judge;
@@ -262,7 +284,8 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
 
   FusedPlan plan;
   const bool fused_ok = h->tm_w_ok && fused_supported(c.dtype, R, c.d, c.V, h->num_sms, &plan);
-  const bool batched_ok = h->tm_w_ok && batched_supported(c.dtype, a->B, c.d, c.V, h->num_sms);
+  const bool fp8 = c.dtype == JD_DTYPE_FP8_E4M3;
+  const bool batched_ok = !fp8 && h->tm_w_ok && batched_supported(c.dtype, a->B, c.d, c.V, h->num_sms);
   int variant = a->variant;
   if (variant == JD_VARIANT_AUTO) {
     if (a->logits_debug) variant = JD_VARIANT_SIMT;
@@ -283,11 +306,15 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   }
   int launches = 0;
   if (a->norm == JD_NORM_RMS) {   // per-row normalisation factors, read by every variant
-    launch_row_scale(cp, h->ws, a->H, c.dtype, st);
+    launch_row_scale(cp, h->ws, a->H, c.dtype == JD_DTYPE_F32 ? JD_DTYPE_F32 : JD_DTYPE_BF16, st);
     launches = 1;
   }
+  if (fp8) {   // rows of H to E4M3 with one scale per row; the judge keeps reading a->H
+    launch_quantize_rows(cp, h->ws, a->H, st);
+    launches += 1;
+  }
   if (variant == JD_VARIANT_SIMT) {
-    launches += run_simt(cp, h->ws, h->W, h->w_judge, a->H, c.dtype, a->logits_debug, st);
+    launches += run_simt(cp, h->ws, h->W, h->w_scale, h->w_judge, a->H, c.dtype, a->logits_debug, st);
   } else if (variant == JD_VARIANT_BATCHED) {
     FusedPlan plan2;   // second pass: B rows through the fused kernel
     if (!fused_supported(c.dtype, a->B, c.d, c.V, h->num_sms, &plan2)) return JD_ERR_UNSUPPORTED;
@@ -301,9 +328,10 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
     launches += n;
   } else {
     CUtensorMap tm_h;
-    if (!make_tensor_map(&tm_h, a->H, (uint64_t)R, (uint64_t)c.d, (uint32_t)plan.n_pad)) return JD_ERR_CUDA;
+    if (!make_tensor_map(&tm_h, fp8 ? (const void*)h->ws.h8 : a->H, (uint64_t)R, (uint64_t)c.d, (uint32_t)plan.n_pad, fp8))
+      return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
-    const int n = run_fused(cp, h->ws, h->tm_w, tm_h, a->H, h->w_judge, plan, st, &err);
+    const int n = run_fused(cp, h->ws, h->tm_w, tm_h, a->H, h->w_judge, plan, st, &err, false, fp8 ? h->w_scale : nullptr);
     if (n < 0) return JD_ERR_CUDA;
     launches += n;
   }

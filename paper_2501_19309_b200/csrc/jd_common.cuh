@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -38,6 +39,8 @@ struct Workspace {
   float* w_sel;        // [maxB][V]  sampling weights (SIMT variant); in the batched variant the selected
                        //            draft rows, tile-major [ceil(V/128)][B][128]
   float* p_sel;        // [maxB][V]  p of the selected row (same)
+  uint8_t* h8;         // [maxR][d] FP8 head: rows of H quantised to E4M3
+  float* h_scale;      // [maxR]    FP8 head: scale of every quantised row
   float* row_scale;    // [maxR] 1 / sqrt(mean square + eps) of every row of H (JD_NORM_RMS)
   int* cnt;            // [maxR] top-K rule: entries of the row that rank above the drafted token
   int* argidx;         // [maxR] top-K rule: lowest token id that attains the row maximum
@@ -110,6 +113,14 @@ __device__ __forceinline__ double warp_sum_double(double v) {
 template <typename T> __device__ __forceinline__ float to_float(T v);
 template <> __device__ __forceinline__ float to_float<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// FP8 E4M3 code (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities).
+struct e4m3_t { uint8_t b; };
+template <> __device__ __forceinline__ float to_float<e4m3_t>(e4m3_t v) {
+  uint32_t h2;   // the hardware conversion widens two codes to two halves; the low one is ours
+  asm("{\n\t.reg .b16 t;\n\tcvt.u16.u32 t, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, t;\n\t}" : "=r"(h2) : "r"((uint32_t)v.b));
+  return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
+}
 
 // ---------------------------------------------------------------------------------------
 // Per-call parameters every kernel family shares.

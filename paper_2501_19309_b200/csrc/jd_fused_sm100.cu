@@ -35,9 +35,10 @@ namespace {
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
 constexpr int kBlockK = 64;                      // bf16 elements per k-slice = one 128-byte swizzle row
+constexpr int kBlockK8 = 128;                    // FP8 codes per k-slice (same 128 bytes)
 constexpr int kWStageBytes = kVocabTile * 128;   // 16 KB
 constexpr int kTmemCols = 512;
-constexpr int kMiscBytes = 16384;                // barriers + reduction scratch at the head of smem
+constexpr int kMiscBytes = 20480;                // barriers + reduction scratch at the head of smem
 constexpr int kMaxStages = 12;
 constexpr int kHStages = 4;
 
@@ -49,6 +50,7 @@ struct FusedParams {
   int tmem_tiles;   // tiles resident in TMEM
   int tile_stride;  // TMEM columns between consecutive tiles (>= rows, multiple of 8, <= N_PAD)
   int R;            // rows of the H matrix given to the MMA: B * (M + 1), or B in sample-only mode
+  int fp8;          // 1: W and H tiles hold FP8 E4M3 codes (128 per 128-byte row), kind::f8f6f4 MMAs
   int sample_only;  // 1: H holds one already selected row per sequence; only the token draw runs
   uint32_t off_h;   // byte offsets inside dynamic smem (from the 1024-aligned base)
   uint32_t off_ovf;
@@ -71,7 +73,8 @@ struct Misc {
   float lse[N_PAD];         // log-normaliser of every row
   float qlse[N_PAD];
   int x_row[N_PAD];         // drafted token of row r (rows j < M), -1 otherwise
-  float scale[N_PAD];       // normalisation factor of the row in TMEM column r (1 without JD_NORM_RMS)
+  float scale[N_PAD];       // factor applied to TMEM column r: RMS normalisation and, for an FP8 head, the row's scale
+  float swt[8][kVocabTile]; // FP8 head: scale of this thread's vocabulary entry in each of the CTA's tiles (else 1)
   int glist[N_PAD];
   // per sequence (B <= N_PAD / 2 in the full mode, B <= N_PAD in sample-only mode)
   int sel_row[N_PAD];
@@ -95,7 +98,7 @@ struct Misc {
 // or from the overflow copy in shared memory
 template <int N_PAD>
 __device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, int ts, uint32_t tmem_lane_base,
-                                            const float* ovf, int tid, const float* sc, float* v0, float* v1) {
+                                            const float* ovf, int tid, const float* sc, const float* swt, float* v0, float* v1) {
   uint32_t a[16], b[16];
 #pragma unroll
   for (int k = 0; k < 16; ++k) { a[k] = 0u; b[k] = 0u; }
@@ -115,16 +118,18 @@ __device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, in
   }
   tmem_wait_ld32(a, b);
 #pragma unroll
+  const float w0 = swt[min(i0, 7) * kVocabTile + tid], w1 = swt[min(i0 + 1, 7) * kVocabTile + tid];
+#pragma unroll
   for (int k = 0; k < 16; ++k) {
-    const float f = sc[c0 + k];   // row normalisation factor (shared memory)
-    v0[k] = __uint_as_float(a[k]) * f;
-    v1[k] = __uint_as_float(b[k]) * f;
+    const float f = sc[c0 + k];   // factor of the row (shared memory)
+    v0[k] = __uint_as_float(a[k]) * (f * w0);
+    v1[k] = __uint_as_float(b[k]) * (f * w1);
   }
 }
 // logits of row r in tiles i0 .. i0+7 (those below T) for this thread's lane, fetched together
 template <int N_PAD>
 __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, int ts, uint32_t tmem_lane_base,
-                                           const float* ovf, int tid, float f, float* out) {
+                                           const float* ovf, int tid, float f, const float* swt, float* out) {
   uint32_t raw[8];
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
@@ -137,7 +142,7 @@ __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, int 
   }
   tmem_wait_ld8(raw);
 #pragma unroll
-  for (int u = 0; u < 8; ++u) out[u] = __uint_as_float(raw[u]) * f;
+  for (int u = 0; u < 8; ++u) out[u] = __uint_as_float(raw[u]) * (f * swt[min(i0 + u, 7) * kVocabTile + tid]);
 }
 
 // Reduces 16 per-lane values over the 32 lanes of a warp with 16 shuffles instead of 80: every
@@ -180,7 +185,7 @@ template <int N_PAD>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, CallParams cp,
                     Workspace ws, const __nv_bfloat16* __restrict__ H, const __nv_bfloat16* __restrict__ wj,
-                    FusedParams fp) {
+                    const float* __restrict__ w_scale, FusedParams fp) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   Misc<N_PAD>& ms = *reinterpret_cast<Misc<N_PAD>*>(smem);
@@ -224,7 +229,15 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     ms.x_row[tid] = x;
     float f = 1.f;   // normalisation factor of the row held in TMEM column tid
     if (cp.norm == JD_NORM_RMS && tid < R) f = ws.row_scale[fp.sample_only ? ws.sel_row[tid] : tid];
+    if (fp.fp8 && tid < R) f *= ws.h_scale[tid];
     ms.scale[tid] = f;
+  }
+  if (tid < kVocabTile) {   // per-vocabulary-row scales of an FP8 head, one per tile of this CTA; 1 otherwise
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int vg = (t0 + u) * kVocabTile + tid;
+      ms.swt[u][tid] = (fp.fp8 && u < T && vg < V) ? __ldg(w_scale + vg) : 1.f;
+    }
   }
   if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ms.tmem_base)),
@@ -247,6 +260,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   if (warp == 4 && lane == 0) {
     // ------------------------------------------------------------------ TMA producer
     const uint64_t pol_w = policy_evict_first(), pol_h = policy_evict_last();
+    const int kelems = fp.fp8 ? kBlockK8 : kBlockK;   // elements per 128-byte k-slice
     int ws_i = 0, hs_i = 0;
     uint32_t wph = 0, hph = 0;
     bool ok = true;
@@ -256,13 +270,13 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         ok = mbar_wait(smem_u32(&ms.empty_h[hs_i]), hph ^ 1u, abort_flag);
         if (!ok) break;
         mbar_expect_tx(smem_u32(&ms.full_h[hs_i]), N_PAD * 128);
-        tma_load_2d(sH + hs_i * (N_PAD * 128), &tmH, smem_u32(&ms.full_h[hs_i]), kb * kBlockK, 0, pol_h);
+        tma_load_2d(sH + hs_i * (N_PAD * 128), &tmH, smem_u32(&ms.full_h[hs_i]), kb * kelems, 0, pol_h);
         if (++hs_i == kHStages) { hs_i = 0; hph ^= 1u; }
         for (int i = g_begin[g]; i < g_end[g]; ++i) {
           ok = mbar_wait(smem_u32(&ms.empty_w[ws_i]), wph ^ 1u, abort_flag);
           if (!ok) break;
           mbar_expect_tx(smem_u32(&ms.full_w[ws_i]), kWStageBytes);
-          tma_load_2d(sW + ws_i * kWStageBytes, &tmW, smem_u32(&ms.full_w[ws_i]), kb * kBlockK, (t0 + i) * kVocabTile,
+          tma_load_2d(sW + ws_i * kWStageBytes, &tmW, smem_u32(&ms.full_w[ws_i]), kb * kelems, (t0 + i) * kVocabTile,
                       pol_w);
           if (++ws_i == fp.stages) { ws_i = 0; wph ^= 1u; }
         }
@@ -271,7 +285,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
   } else if (warp == 5 && lane == 0) {
     // ------------------------------------------------------------------ MMA issuer
-    const uint32_t idesc = make_idesc(N_PAD);
+    const uint32_t idesc = fp.fp8 ? make_idesc_e4m3(N_PAD) : make_idesc(N_PAD);
     int ws_i = 0, hs_i = 0;
     uint32_t wph = 0, hph = 0;
     bool ok = true;
@@ -293,9 +307,11 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           const uint32_t wb = sW + ws_i * kWStageBytes;
           const uint32_t dcol = tmem_base + (uint32_t)((i - g_begin[g]) * fp.tile_stride);
 #pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k) {
-            umma_bf16(dcol, make_smem_desc(wb + k * 32), make_smem_desc(hb + k * 32), idesc,
-                      (kb > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < 4; ++k) {   // four MMAs of 32 bytes of K each: 16 bf16 or 32 FP8 codes
+            const uint64_t da = make_smem_desc(wb + k * 32), db = make_smem_desc(hb + k * 32);
+            const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+            if (fp.fp8) umma_e4m3(dcol, da, db, idesc, acc);
+            else umma_bf16(dcol, da, db, idesc, acc);
           }
           umma_commit(smem_u32(&ms.empty_w[ws_i]));
           if (++ws_i == fp.stages) { ws_i = 0; wph ^= 1u; }
@@ -418,7 +434,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         const int r = ms.glist[e], x = ms.x_row[r];
         const int i = x / kVocabTile - t0;
         float one[8];
-        load_cols8<N_PAD>(i, i + 1, r, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[r], one);
+        load_cols8<N_PAD>(i, i + 1, r, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[r], &ms.swt[0][0], one);
         if (tid == (x % kVocabTile)) ws.gath[r] = one[0];
       }
     }
@@ -430,7 +446,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (ok) {
         for (int i0 = 0; i0 < T; i0 += 2) {
           float v0[16], v1[16];
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0], v0, v1);
           const bool val0 = (t0 + i0) * kVocabTile + tid < V;
           const bool val1 = (i0 + 1 < T) && ((t0 + i0 + 1) * kVocabTile + tid < V);
           if (val0) {
@@ -459,7 +475,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (ok) {
         for (int i0 = 0; i0 < T; i0 += 2) {
           float v0[16], v1[16];
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0], v0, v1);
           const bool val0 = (t0 + i0) * kVocabTile + tid < V;
           const bool val1 = (i0 + 1 < T) && ((t0 + i0 + 1) * kVocabTile + tid < V);
           if (val0) {
@@ -515,7 +531,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
         for (int i0 = 0; i0 < T; i0 += 2) {
           float v0[16], v1[16];
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0], v0, v1);
           const int vg0 = (t0 + i0) * kVocabTile + tid, vg1 = vg0 + kVocabTile;
           const bool val0 = vg0 < V, val1 = (i0 + 1 < T) && vg1 < V;
 #pragma unroll
@@ -692,7 +708,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             d0[k] = __ldg(base0 + kk * kVocabTile);
             d1[k] = __ldg(base1 + kk * kVocabTile);
           }
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, v0, v1);
+          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0], v0, v1);
 #pragma unroll
           for (int k = 0; k < 16; ++k) {
             const float p0 = fast_exp2(fmaf(v0[k], kLog2e, -lp2[k])), q0 = fast_exp2(fmaf(d0[k], kLog2e, -lq2[k]));
@@ -737,7 +753,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           for (int q = 0; q < 4; ++q) {
             const int b = min(b0 + q, cp.B - 1);
             const int col = fp.sample_only ? b : ms.sel_row[b];   // TMEM column of this sequence's selected row
-            load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], lg[q]);
+            load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], &ms.swt[0][0], lg[q]);
           }
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -875,7 +891,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                                               : dlrow + vg;
             dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(src) : 0.f;
           }
-          load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], lg);
+          load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], &ms.swt[0][0], lg);
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
@@ -951,14 +967,14 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
 template <int N_PAD>
 cudaError_t launch_fused(const CUtensorMap& tmW, const CUtensorMap& tmH, const CallParams& cp, const Workspace& ws,
-                         const void* H, const void* wj, const FusedParams& fp, const FusedPlan& plan,
-                         cudaStream_t st) {
+                         const void* H, const void* wj, const float* w_scale, const FusedParams& fp,
+                         const FusedPlan& plan, cudaStream_t st) {
   auto kern = fused_verify_kernel<N_PAD>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (e != cudaSuccess) return e;
   const __nv_bfloat16* Hp = (const __nv_bfloat16*)H;
   const __nv_bfloat16* wp = (const __nv_bfloat16*)wj;
-  void* args[] = {(void*)&tmW, (void*)&tmH, (void*)&cp, (void*)&ws, (void*)&Hp, (void*)&wp, (void*)&fp};
+  void* args[] = {(void*)&tmW, (void*)&tmH, (void*)&cp, (void*)&ws, (void*)&Hp, (void*)&wp, (void*)&w_scale, (void*)&fp};
   return cudaLaunchCooperativeKernel((const void*)kern, dim3(plan.num_ctas), dim3(kThreads), args, plan.smem_bytes,
                                      st);
 }
@@ -966,7 +982,10 @@ cudaError_t launch_fused(const CUtensorMap& tmW, const CUtensorMap& tmH, const C
 }  // namespace
 
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan) {
-  if (dtype != JD_DTYPE_BF16 || d % kBlockK != 0 || d < kBlockK || R < 1 || R > 96) return false;
+  const bool fp8 = dtype == JD_DTYPE_FP8_E4M3;
+  if (dtype != JD_DTYPE_BF16 && !fp8) return false;
+  const int kelems = fp8 ? kBlockK8 : kBlockK;
+  if (d % kelems != 0 || d < kelems || R < 1 || R > 96) return false;
   if (num_sms < 1 || num_sms > kMaxCtas) return false;
   const int n_pad = (R + 15) / 16 * 16;
   const int num_tiles = (V + kVocabTile - 1) / kVocabTile;
@@ -979,10 +998,11 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
   const int tmem_tiles = std::min(max_tiles, (kTmemCols - n_pad) / stride + 1);
   const int n_ovf = max_tiles - tmem_tiles;
   if (n_ovf > tmem_tiles) return false;   // the overflow group itself must fit in TMEM
+  if (fp8 && max_tiles > 8) return false;  // the per-tile vocabulary scales are kept for eight tiles
   const size_t fixed = 1024 /*alignment slack*/ + kMiscBytes + (size_t)kHStages * n_pad * 128 +
                        (size_t)n_ovf * kVocabTile * n_pad * 4;
   const size_t budget = 227 * 1024;
-  if (fixed + 4 * (size_t)kWStageBytes > budget) return false;
+  if (fixed + 3 * (size_t)kWStageBytes > budget) return false;   // at least a three-deep W ring
   int stages = (int)((budget - fixed) / kWStageBytes);
   stages = std::min(stages, kMaxStages);
   if (plan) {
@@ -999,9 +1019,10 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
 
 int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
               const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err,
-              bool sample_only) {
+              bool sample_only, const float* w_scale_fp8) {
   FusedParams fp;
-  fp.num_kb = cp.d / kBlockK;
+  fp.fp8 = w_scale_fp8 ? 1 : 0;
+  fp.num_kb = cp.d / (fp.fp8 ? kBlockK8 : kBlockK);
   fp.num_tiles = (cp.V + kVocabTile - 1) / kVocabTile;
   fp.stages = plan.stages;
   fp.tmem_tiles = plan.tmem_tiles;
@@ -1015,12 +1036,12 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
   fp.off_w = (fp.off_w + 1023u) & ~1023u;
   cudaError_t e;
   switch (plan.n_pad) {
-    case 16: e = launch_fused<16>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
-    case 32: e = launch_fused<32>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
-    case 48: e = launch_fused<48>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
-    case 64: e = launch_fused<64>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
-    case 80: e = launch_fused<80>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
-    case 96: e = launch_fused<96>(tmW, tmH, cp, ws, H, w_judge, fp, plan, st); break;
+    case 16: e = launch_fused<16>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 32: e = launch_fused<32>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 48: e = launch_fused<48>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 64: e = launch_fused<64>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 80: e = launch_fused<80>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 96: e = launch_fused<96>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
     default: e = cudaErrorInvalidValue; break;
   }
   *err = e;

@@ -8,10 +8,12 @@
 namespace jd {
 
 // CUDA-core pipeline (jd_simt.cu). Each returns after enqueueing on `st`.
-int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const void* w_judge, const void* H, int dtype,
+int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const float* w_scale, const void* w_judge,
+             const void* H, int dtype,
              float* logits_debug, cudaStream_t st);
 int launch_q_stats(const CallParams& cp, const Workspace& ws, cudaStream_t st);   // returns partials per draft row
 void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, const void* w, int dtype, cudaStream_t st);
+void launch_quantize_rows(const CallParams& cp, const Workspace& ws, const void* H_bf16, cudaStream_t st);
 void launch_row_scale(const CallParams& cp, const Workspace& ws, const void* H, int dtype, cudaStream_t st);
 void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st);
 void launch_decide(const CallParams& cp, const Workspace& ws, cudaStream_t st);
@@ -33,7 +35,7 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
 // Returns the number of kernels launched, or -1 with *err set.
 int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
               const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err,
-              bool sample_only = false);
+              bool sample_only = false, const float* w_scale_fp8 = nullptr);
 
 // Two-pass tensor-core variant for many rows (jd_batched_sm100.cu). tmW256 / tmW128: W with
 // 256- and 128-row boxes; tmH: H with a 128-row box; tmHsel: the handle's [B, d] gather buffer

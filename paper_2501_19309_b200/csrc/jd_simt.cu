@@ -23,7 +23,8 @@ constexpr int kSimtK = 32;
 template <typename T, int kMode>
 __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, Workspace ws, const T* __restrict__ W,
                                                                  const T* __restrict__ H, int R, int np,
-                                                                 float* __restrict__ logits_debug) {
+                                                                 float* __restrict__ logits_debug,
+                                                                 const float* __restrict__ w_scale) {
   __shared__ float sW[kVocabTile][kSimtK + 1];
   __shared__ __align__(16) float sH[kSimtRows][kSimtK];
   __shared__ float s_m[4][kSimtRows], s_s[4][kSimtRows];
@@ -42,6 +43,7 @@ __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, 
     const int r = r0 + tid;
     s_row[tid] = (r < R) ? (kSample ? ws.sel_row[r] : r) : -1;
     s_scale[tid] = (cp.norm == JD_NORM_RMS && s_row[tid] >= 0) ? ws.row_scale[s_row[tid]] : 1.f;
+    if (w_scale && s_row[tid] >= 0) s_scale[tid] *= ws.h_scale[s_row[tid]];   // FP8 head: scale of the quantised row
   }
   __syncthreads();
 
@@ -79,6 +81,11 @@ __global__ void __launch_bounds__(kVocabTile) simt_logits_kernel(CallParams cp, 
 
 #pragma unroll
   for (int i = 0; i < kSimtRows; ++i) acc[i] *= s_scale[i];   // 1 when no normalisation is asked for
+  if (w_scale) {   // FP8 head: scale of this thread's vocabulary row
+    const float sv = v < V ? w_scale[v] : 0.f;
+#pragma unroll
+    for (int i = 0; i < kSimtRows; ++i) acc[i] *= sv;
+  }
 
   const bool valid_v = v < V;
   if (kMode == 2) {
@@ -199,6 +206,40 @@ __global__ void __launch_bounds__(256) q_stats_kernel(CallParams cp, Workspace w
       if (x < 0 || x >= V) { set_status(ws.status, JD_ERR_BAD_TOKEN); x = min(max(x, 0), V - 1); }
       ws.qgath[bm] = row[x];
     }
+  }
+}
+
+// FP8 head: quantises every row of H to E4M3 with one scale per row, s = amax / 448 and
+// code = e4m3(h * (448 / amax)), round to nearest even, saturating; all in float32.
+__global__ void __launch_bounds__(256) quantize_rows_kernel(CallParams cp, Workspace ws,
+                                                            const __nv_bfloat16* __restrict__ H) {
+  __shared__ float s_p[8];
+  __shared__ float s_amax;
+  const int row = blockIdx.x;
+  const __nv_bfloat16* h = H + (size_t)row * cp.d;
+  float amax = 0.f;
+  for (int k = threadIdx.x; k < cp.d; k += blockDim.x) amax = fmaxf(amax, fabsf(__bfloat162float(h[k])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if ((threadIdx.x & 31) == 0) s_p[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < 8; ++i) t = fmaxf(t, s_p[i]);
+    s_amax = t;
+    ws.h_scale[row] = __fdiv_rn(t, 448.f);
+  }
+  __syncthreads();
+  amax = s_amax;
+  const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+  uint8_t* out = ws.h8 + (size_t)row * cp.d;
+  for (int k = 2 * threadIdx.x; k < cp.d; k += 2 * blockDim.x) {
+    const float a = __fmul_rn(__bfloat162float(h[k]), inv);
+    const float b = k + 1 < cp.d ? __fmul_rn(__bfloat162float(h[k + 1]), inv) : 0.f;
+    unsigned short pair;   // upper byte = code of the first operand, lower byte = code of the second
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair) : "f"(b), "f"(a));
+    out[k] = (uint8_t)(pair & 0xFF);
+    if (k + 1 < cp.d) out[k + 1] = (uint8_t)(pair >> 8);
   }
 }
 
@@ -367,6 +408,10 @@ void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, cons
     judge_dot_kernel<float><<<cp.B * cp.M, 256, 0, st>>>(cp, ws, (const float*)H, (const float*)w);
 }
 
+void launch_quantize_rows(const CallParams& cp, const Workspace& ws, const void* H_bf16, cudaStream_t st) {
+  quantize_rows_kernel<<<cp.B * (cp.M + 1), 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H_bf16);
+}
+
 void launch_row_scale(const CallParams& cp, const Workspace& ws, const void* H, int dtype, cudaStream_t st) {
   const int R = cp.B * (cp.M + 1);
   if (dtype == JD_DTYPE_BF16) row_scale_kernel<__nv_bfloat16><<<R, 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H);
@@ -388,27 +433,28 @@ void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream
 
 template <typename T>
 static void simt_logits(const CallParams& cp, const Workspace& ws, const void* W, const void* H, int mode, int np,
-                        float* logits_debug, cudaStream_t st) {
+                        float* logits_debug, const float* w_scale, cudaStream_t st) {
   const int R = mode == 1 ? cp.B : cp.B * (cp.M + 1);
   dim3 grid(np, (R + kSimtRows - 1) / kSimtRows);
   if (mode == 1)
-    simt_logits_kernel<T, 1><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, nullptr);
+    simt_logits_kernel<T, 1><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, nullptr, w_scale);
   else if (mode == 2)
-    simt_logits_kernel<T, 2><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, nullptr);
+    simt_logits_kernel<T, 2><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, nullptr, w_scale);
   else
-    simt_logits_kernel<T, 0><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, logits_debug);
+    simt_logits_kernel<T, 0><<<grid, kVocabTile, 0, st>>>(cp, ws, (const T*)W, (const T*)H, R, np, logits_debug, w_scale);
 }
 
-int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const void* w_judge, const void* H, int dtype,
-             float* logits_debug, cudaStream_t st) {
+int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const float* w_scale, const void* w_judge,
+             const void* H, int dtype, float* logits_debug, cudaStream_t st) {
   const int np = (cp.V + kVocabTile - 1) / kVocabTile;
-  const bool bf = dtype == JD_DTYPE_BF16;
   auto logits = [&](int mode, float* dbg) {
-    if (bf) simt_logits<__nv_bfloat16>(cp, ws, W, H, mode, np, dbg, st);
-    else simt_logits<float>(cp, ws, W, H, mode, np, dbg, st);
+    if (dtype == JD_DTYPE_FP8_E4M3)   // E4M3 weights against the E4M3 rows the caller quantised into ws.h8
+      simt_logits<e4m3_t>(cp, ws, W, ws.h8, mode, np, dbg, w_scale, st);
+    else if (dtype == JD_DTYPE_BF16) simt_logits<__nv_bfloat16>(cp, ws, W, H, mode, np, dbg, nullptr, st);
+    else simt_logits<float>(cp, ws, W, H, mode, np, dbg, nullptr, st);
   };
   const int nq = launch_q_stats(cp, ws, st);
-  launch_judge(cp, ws, H, w_judge, dtype, st);
+  launch_judge(cp, ws, H, w_judge, dtype == JD_DTYPE_F32 ? JD_DTYPE_F32 : JD_DTYPE_BF16, st);
   logits(0, logits_debug);
   launch_fold(cp, ws, np, nq, st);
   if (cp.rule == JD_RULE_TOPK) {   // ranks and argmax need the folded maxima; the decision writes the token

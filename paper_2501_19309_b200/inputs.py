@@ -49,7 +49,8 @@ class Workload:
     M: int
     d: int
     V: int
-    dtype: str = "bf16"            # "bf16" or "f32": storage type of W, H, w_judge
+    dtype: str = "bf16"            # "bf16" or "f32": storage type of W, H, w_judge; "fp8": W is FP8 E4M3
+                                   # codes with one float32 scale per vocabulary row, H and w_judge bf16
     alpha: float = 4.0             # planted-alignment scale (used when alpha_range is None)
     alpha_range: Optional[tuple] = None   # (lo, hi): alpha ~ U[lo, hi]
     alpha_per: str = "seq"         # "seq": one alpha per sequence, "row": one per H row
@@ -86,7 +87,7 @@ CONFIGS = {
 class Inputs:
     wl: Workload
     data_seed: int
-    W: np.ndarray             # [V, d] uint16 (bf16 bits) or float32
+    W: np.ndarray             # [V, d] uint16 (bf16 bits), float32, or uint8 (FP8 E4M3 codes, dtype "fp8")
     H: np.ndarray             # [B, M+1, d] same storage type as W
     w_judge: np.ndarray       # [d] same storage type as W
     b_judge: float
@@ -95,6 +96,7 @@ class Inputs:
     draft_logits: np.ndarray  # [B, M, V] float32
     seed: int                 # seed handed to the verify call's counter-based RNG
     planted_tokens: np.ndarray  # [B, M+1] int32: token whose W row each H row leans to
+    w_scale: Optional[np.ndarray] = None   # [V] float32 row scales of an FP8 head (dtype "fp8")
 
 
 def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
@@ -114,6 +116,23 @@ def as_f32(a: np.ndarray) -> np.ndarray:
     return bf16_bits_to_f32(a) if a.dtype == np.uint16 else np.asarray(a, dtype=np.float32)
 
 
+def quantise_rows_fp8(a32: np.ndarray):
+    """Per-row FP8 E4M3 storage of a float32 matrix: (codes uint8, scale float32) with
+    a ~ scale[:, None] * e4m3(codes); scale = row amax / 448. The float -> E4M3 rounding is
+    PyTorch's CPU conversion (nearest, ties to even)."""
+    import torch
+    a32 = np.ascontiguousarray(a32, dtype=np.float32)
+    amax = np.abs(a32).max(axis=1).astype(np.float32)
+    scale = (np.where(amax > 0, amax, np.float32(1.0)) / np.float32(448.0)).astype(np.float32)
+    q = torch.from_numpy(a32 / scale[:, None]).clamp_(-448.0, 448.0).to(torch.float8_e4m3fn)
+    return q.view(torch.uint8).numpy(), scale
+
+
+def fp8_codes_to_f32(codes: np.ndarray) -> np.ndarray:
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(codes)).view(torch.float8_e4m3fn).float().numpy()
+
+
 def _gen(wl: Workload, data_seed: int, stream: int) -> np.random.Generator:
     return np.random.Generator(np.random.Philox(key=[1000 * wl.config_id + data_seed, stream]))
 
@@ -124,6 +143,8 @@ def _store(a32: np.ndarray, dtype: str) -> np.ndarray:
 
 def make_W_rows(wl: Workload, data_seed: int, row_lo: int, row_hi: int) -> np.ndarray:
     """Rows [row_lo, row_hi) of W in storage type; rows are N(0, 1/d) rounded to dtype."""
+    if wl.dtype == "fp8":
+        raise ValueError("FP8 heads are built by make_inputs (codes + row scales)")
     out = np.empty((row_hi - row_lo, wl.d), dtype=np.uint16 if wl.dtype == "bf16" else np.float32)
     scale = np.float32(1.0 / np.sqrt(wl.d))
     blk_lo = row_lo // W_BLOCK_ROWS
@@ -163,7 +184,20 @@ def make_inputs(wl: Workload, data_seed: int = 0, W: Optional[np.ndarray] = None
     """Draw one workload.  ``W`` may be passed in when it was already generated
     for this (workload, data_seed); it is not checked."""
     B, M, d, V = wl.B, wl.M, wl.d, wl.V
-    if W is None:
+    w_scale = None
+    if wl.dtype == "fp8":
+        # the same N(0, 1/d) head as the bf16 workload, stored as FP8 E4M3 with a scale per row
+        if W is None:
+            base = dataclasses.replace(wl, dtype="f32")
+            codes = np.empty((V, d), dtype=np.uint8)
+            w_scale = np.empty(V, dtype=np.float32)
+            for r0 in range(0, V, 8 * W_BLOCK_ROWS):
+                r1 = min(V, r0 + 8 * W_BLOCK_ROWS)
+                codes[r0:r1], w_scale[r0:r1] = quantise_rows_fp8(make_W_rows(base, data_seed, r0, r1))
+            W = codes
+        else:
+            W, w_scale = W
+    elif W is None:
         W = make_W(wl, data_seed)
 
     g = _gen(wl, data_seed, _S_TOKENS)
@@ -185,14 +219,18 @@ def make_inputs(wl: Workload, data_seed: int = 0, W: Optional[np.ndarray] = None
     gj = _gen(wl, data_seed, _S_JUDGE)
     w32 = gj.standard_normal(d, dtype=np.float32) * np.float32(1.0 / np.sqrt(d))
     b_judge = float(gj.standard_normal() * wl.b_judge_std) if wl.b_judge_std > 0 else 0.0
-    w_store = _store(w32, wl.dtype)
+    act_dtype = "bf16" if wl.dtype == "fp8" else wl.dtype     # storage type of H and w_judge
+    w_store = _store(w32, act_dtype)
     w_val = as_f32(w_store).astype(np.float64)
 
     # H = alpha * unit(W[planted]) + sigma * noise, rounded to the storage type
     gn = _gen(wl, data_seed, _S_NOISE)
     H32 = np.empty((B, M + 1, d), dtype=np.float32)
     for b in range(B):
-        rows = as_f32(W[planted[b]]).astype(np.float64)                 # [M+1, d]
+        if wl.dtype == "fp8":
+            rows = (fp8_codes_to_f32(W[planted[b]]) * w_scale[planted[b]][:, None]).astype(np.float64)
+        else:
+            rows = as_f32(W[planted[b]]).astype(np.float64)             # [M+1, d]
         unit = rows / np.linalg.norm(rows, axis=1, keepdims=True)
         noise = gn.standard_normal((M + 1, d), dtype=np.float32).astype(np.float64) * wl.sigma
         H32[b] = (alpha[b][:, None].astype(np.float64) * unit + noise).astype(np.float32)
@@ -223,7 +261,7 @@ def make_inputs(wl: Workload, data_seed: int = 0, W: Optional[np.ndarray] = None
     bi, ji = np.meshgrid(np.arange(B), np.arange(M), indexing="ij")
     dl[bi, ji, draft_tokens] += boost
 
-    H = _store(H32, wl.dtype)
+    H = _store(H32, act_dtype)
     return Inputs(wl=wl, data_seed=data_seed, W=W, H=H, w_judge=w_store, b_judge=b_judge,
                   tau=wl.tau if tau is None else tau, draft_tokens=draft_tokens,
-                  draft_logits=np.ascontiguousarray(dl), seed=data_seed, planted_tokens=planted)
+                  draft_logits=np.ascontiguousarray(dl), seed=data_seed, planted_tokens=planted, w_scale=w_scale)

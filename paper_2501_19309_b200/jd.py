@@ -19,7 +19,7 @@ _lib = None
 
 JD_OK, JD_ERR_INVALID_ARG, JD_ERR_UNSUPPORTED, JD_ERR_ARCH = 0, 1, 2, 3
 JD_ERR_ALLOC, JD_ERR_CUDA, JD_ERR_TIMEOUT, JD_ERR_BAD_TOKEN = 4, 5, 6, 7
-JD_DTYPE_F32, JD_DTYPE_BF16 = 0, 1
+JD_DTYPE_F32, JD_DTYPE_BF16, JD_DTYPE_FP8_E4M3 = 0, 1, 2
 JD_MODE_STANDARD, JD_MODE_JUDGE, JD_MODE_JUDGE_OR_STANDARD = 0, 1, 2
 JD_RESAMPLE_RESIDUAL, JD_RESAMPLE_TARGET_P = 0, 1
 JD_VARIANT_AUTO, JD_VARIANT_SIMT, JD_VARIANT_FUSED, JD_VARIANT_BATCHED = 0, 1, 2, 3
@@ -33,7 +33,7 @@ VARIANTS = {"auto": JD_VARIANT_AUTO, "simt": JD_VARIANT_SIMT, "fused": JD_VARIAN
 
 EXPORTS = ["jd_version", "jd_status_string", "jd_workspace_bytes", "jd_create", "jd_destroy", "jd_set_head",
            "jd_verify", "jd_verify_host", "jd_last_device_status", "jd_last_launch_info", "jd_philox_uniforms",
-           "jd_verify_static"]
+           "jd_verify_static", "jd_set_head_fp8"]
 
 
 class jd_config_t(C.Structure):
@@ -77,6 +77,7 @@ def load():
     lib.jd_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(jd_config_t)]
     lib.jd_destroy.argtypes = [C.c_void_p]
     lib.jd_set_head.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
+    lib.jd_set_head_fp8.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
     lib.jd_verify.argtypes = [C.c_void_p, C.POINTER(jd_verify_args_t), C.c_void_p]
     lib.jd_verify_host.argtypes = [C.c_void_p, C.POINTER(jd_verify_args_t), C.c_void_p]
     lib.jd_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_int)]
@@ -119,6 +120,11 @@ def jd_destroy(h) -> None:
 
 def jd_set_head(h, W_ptr: int, w_judge_ptr: int, b_judge: float) -> int:
     return load().jd_set_head(h, C.c_void_p(W_ptr), C.c_void_p(w_judge_ptr), C.c_float(b_judge))
+
+
+def jd_set_head_fp8(h, W8_ptr: int, w_scale_ptr: int, w_judge_ptr: int, b_judge: float) -> int:
+    return load().jd_set_head_fp8(h, C.c_void_p(W8_ptr), C.c_void_p(w_scale_ptr), C.c_void_p(w_judge_ptr),
+                                  C.c_float(b_judge))
 
 
 def jd_verify(h, args: jd_verify_args_t, stream_ptr: int = 0) -> int:
@@ -169,8 +175,10 @@ class Verifier:
     def __init__(self, max_B: int, max_M: int, d: int, V: int, dtype: str = "bf16", device: int = 0):
         import torch
         self.torch = torch
-        self.cfg = jd_config_t(max_B, max_M, d, V, JD_DTYPE_BF16 if dtype == "bf16" else JD_DTYPE_F32, device)
-        self.dtype = torch.bfloat16 if dtype == "bf16" else torch.float32
+        code = {"bf16": JD_DTYPE_BF16, "f32": JD_DTYPE_F32, "fp8": JD_DTYPE_FP8_E4M3}[dtype]
+        self.cfg = jd_config_t(max_B, max_M, d, V, code, device)
+        self.fp8 = dtype == "fp8"
+        self.dtype = torch.float32 if dtype == "f32" else torch.bfloat16     # type of H and w_judge
         self.device = torch.device("cuda", device)
         self.h = jd_create(self.cfg)
         self._W = self._w = None
@@ -186,10 +194,20 @@ class Verifier:
         except Exception:
             pass
 
-    def set_head(self, W, w_judge, b_judge: float) -> None:
-        assert W.is_cuda and W.dtype == self.dtype and W.is_contiguous() and tuple(W.shape) == (self.cfg.V, self.cfg.d)
+    def set_head(self, W, w_judge, b_judge: float, w_scale=None) -> None:
+        """W: [V, d] in the handle's dtype; for an FP8 head W holds uint8 E4M3 codes and w_scale [V]
+        (float32) is required."""
+        t = self.torch
+        assert W.is_cuda and W.is_contiguous() and tuple(W.shape) == (self.cfg.V, self.cfg.d)
         assert w_judge.is_cuda and w_judge.dtype == self.dtype and w_judge.is_contiguous()
-        self._W, self._w = W, w_judge         # keep the borrowed tensors alive
+        self._W, self._w, self._ws = W, w_judge, w_scale         # keep the borrowed tensors alive
+        if self.fp8:
+            assert W.dtype == t.uint8 and w_scale is not None and w_scale.dtype == t.float32 and w_scale.is_cuda
+            st = jd_set_head_fp8(self.h, W.data_ptr(), w_scale.data_ptr(), w_judge.data_ptr(), float(b_judge))
+            if st != JD_OK:
+                raise JdError(st, "jd_set_head_fp8")
+            return
+        assert W.dtype == self.dtype
         st = jd_set_head(self.h, W.data_ptr(), w_judge.data_ptr(), float(b_judge))
         if st != JD_OK:
             raise JdError(st, "jd_set_head")

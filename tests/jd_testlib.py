@@ -40,7 +40,8 @@ def upload(inp: I.Inputs, device="cuda:0"):
             t = t.view(torch.bfloat16)
         return t.to(device)
 
-    return dict(W=store(inp.W), H=store(inp.H), w=store(inp.w_judge),
+    ws = None if inp.w_scale is None else torch.from_numpy(inp.w_scale).to(device)
+    return dict(W=store(inp.W), H=store(inp.H), w=store(inp.w_judge), w_scale=ws,
                 x=torch.from_numpy(inp.draft_tokens).to(device),
                 dl=torch.from_numpy(inp.draft_logits).to(device))
 
@@ -49,7 +50,7 @@ def make_verifier(inp: I.Inputs, dev: dict, max_B=None, max_M=None):
     from paper_2501_19309_b200 import jd
     wl = inp.wl
     v = jd.Verifier(max_B or wl.B, max_M or wl.M, wl.d, wl.V, wl.dtype)
-    v.set_head(dev["W"], dev["w"], inp.b_judge)
+    v.set_head(dev["W"], dev["w"], inp.b_judge, w_scale=dev.get("w_scale"))
     return v
 
 
@@ -64,7 +65,7 @@ def run_oracle(inp: I.Inputs, mode, seed=None, tau=None, resample="residual", se
     return O.jd_oracle_verify(inp.W, inp.w_judge, inp.b_judge, inp.H, inp.draft_tokens, inp.draft_logits,
                               inp.tau if tau is None else tau, inp.seed if seed is None else seed,
                               mode, resample, sequences=sequences, keep_logits=keep_logits, rule=rule, top_k=top_k,
-                              rms_eps=rms_eps)
+                              rms_eps=rms_eps, w_scale=inp.w_scale)
 
 
 @dataclasses.dataclass

@@ -359,3 +359,42 @@ def test_rms_norm_makes_target_side_scale_invariant_on_device():
     assert np.array_equal(a["accept_len"], b["accept_len"]) and np.array_equal(a["masks"] & 1, b["masks"] & 1)
     assert not np.allclose(a["judge_scores"], b["judge_scores"])     # the judge reads the raw rows
     ver.close()
+
+
+# ------------------------------------------------------------------ FP8 E4M3 head
+FP8_CASES = [
+    ("simt", 2, 5, 100, 515),
+    ("simt", 3, 4, 256, 1300),
+    ("fused", 1, 8, 256, 128256),
+    ("fused", 4, 16, 128, 40000 + 77),
+    ("fused", 1, 25, 512, 128256),
+    ("fused", 6, 15, 128, 128256),            # overflow tiles
+]
+
+
+@pytest.mark.parametrize("variant,B,M,d,V", FP8_CASES)
+def test_fp8_head_parity(variant, B, M, d, V):
+    wl = I.CONFIGS[2].scaled("fp8-%s-%d-%d-%d-%d" % (variant, B, M, d, V), B=B, M=M, d=d, V=V, dtype="fp8")
+    rep = run_case(wl, 13, variant=variant, modes=("judge_or_standard", "standard"), seeds=[0, 1],
+                   expect_variant=variant, check_logits=(variant == "simt"))
+    assert rep.sequences == 4 * B
+    if variant == "fused":
+        run_case(wl, 13, variant=variant, modes=("standard",), seeds=[0], rule="greedy", rms_eps=1e-5)
+
+
+def test_fp8_fused_matches_fp8_simt_and_row_codes_match_checker():
+    from oracle import jd_oracle as O
+    wl = I.CONFIGS[2].scaled("fp8x", B=4, M=16, d=256, V=128256, dtype="fp8")
+    inp = I.make_inputs(wl, 2)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    a = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 1, "judge_or_standard", variant="fused"))
+    b = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 1, "judge_or_standard", variant="simt"))
+    assert np.array_equal(a["accept_len"], b["accept_len"]) and np.array_equal(a["masks"], b["masks"])
+    assert np.allclose(a["row_lse"], b["row_lse"], rtol=0, atol=1e-4)
+    # an FP8 handle refuses the bf16 registration call and the batched variant
+    from paper_2501_19309_b200 import jd
+    assert jd.jd_set_head(ver.h, dev["W"].data_ptr(), dev["w"].data_ptr(), 0.0) == jd.JD_ERR_INVALID_ARG
+    args, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, variant="batched")
+    assert jd.jd_verify(ver.h, args) == jd.JD_ERR_UNSUPPORTED
+    ver.close()

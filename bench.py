@@ -110,7 +110,10 @@ def aggregate_value(units_per_rank_step: int, steps: int, world: int, max_second
 
 
 def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, which: str) -> dict:
-    bytes_alg = wl.V * wl.d * 2 + wl.R * wl.d * 2            # W once + H once
+    if wl.dtype == "fp8":   # one byte per weight + a float per vocabulary row; H read as bf16 once
+        bytes_alg = wl.V * wl.d + wl.V * 4 + wl.R * wl.d * 2
+    else:
+        bytes_alg = wl.V * wl.d * 2 + wl.R * wl.d * 2        # W once + H once
     flops = 2.0 * wl.R * wl.V * wl.d
     tf_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     t_bytes = bytes_alg / (peaks["hbm_gbs"] * 1e9)
@@ -181,13 +184,15 @@ def run_reference(args, wl) -> None:
 def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     """Times K device-resident calls and K_e2e host-buffer calls of one workload on this rank."""
     inp = I.make_inputs(wl, data_seed)
-    W = torch.from_numpy(inp.W).view(torch.bfloat16).to(device)
+    fp8 = wl.dtype == "fp8"
+    W = torch.from_numpy(inp.W).to(device) if fp8 else torch.from_numpy(inp.W).view(torch.bfloat16).to(device)
+    w_scale = torch.from_numpy(inp.w_scale).to(device) if fp8 else None
     H = torch.from_numpy(inp.H).view(torch.bfloat16).to(device)
     w = torch.from_numpy(inp.w_judge).view(torch.bfloat16).to(device)
     x = torch.from_numpy(inp.draft_tokens).to(device)
     dl = torch.from_numpy(inp.draft_logits).to(device)
-    ver = jd.Verifier(wl.B, wl.M, wl.d, wl.V, "bf16", device.index)
-    ver.set_head(W, w, inp.b_judge)
+    ver = jd.Verifier(wl.B, wl.M, wl.d, wl.V, "fp8" if fp8 else "bf16", device.index)
+    ver.set_head(W, w, inp.b_judge, w_scale=w_scale)
     out = ver.alloc_outputs(wl.B, wl.M)
     a_args = [ver.make_args(H, x, dl, inp.tau, s, "judge_or_standard", out=out)[0] for s in range(8)]
     stream = torch.cuda.current_stream(device)
@@ -269,7 +274,8 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, help="workload id of the headline line (1..4)")
-    ap.add_argument("--others", default="2,3,4", help="comma list of further workloads summarised in the same line")
+    ap.add_argument("--others", default="2,3,4,3f", help="comma list of further workloads summarised in the same "
+                    "line; a trailing f = the same shape with an FP8 E4M3 head")
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -307,10 +313,14 @@ def main() -> None:
     if rank == 0 and args.others:
         small = argparse.Namespace(**vars(args))
         small.dist = False
-        for cid in [int(c) for c in args.others.split(",") if c.strip()]:
-            if cid == args.config or cid not in I.CONFIGS:
+        for tok in [c.strip() for c in args.others.split(",") if c.strip()]:
+            as_fp8 = tok.endswith("f")
+            cid = int(tok.rstrip("f"))
+            if (cid == args.config and not as_fp8) or cid not in I.CONFIGS:
                 continue
             owl = I.CONFIGS[cid]
+            if as_fp8:
+                owl = owl.scaled(owl.name + "-fp8", dtype="fp8")
             small.steps = max(50, min(args.steps, 300))
             small.e2e_steps = 10
             r = measure_workload(owl, small, torch, jd, device, data_seed=0, sample_clocks=False)

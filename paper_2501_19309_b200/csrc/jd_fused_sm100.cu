@@ -181,7 +181,9 @@ __device__ __forceinline__ int reduce16_index(int lane) {
   return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
 }
 
-template <int N_PAD>
+// kFp8 is a template parameter, not a runtime flag: a kernel whose MMA loop can reach both
+// tcgen05.mma kinds ran its bf16 main loop 40 % slower.
+template <int N_PAD, bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, CallParams cp,
                     Workspace ws, const __nv_bfloat16* __restrict__ H, const __nv_bfloat16* __restrict__ wj,
@@ -285,7 +287,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
   } else if (warp == 5 && lane == 0) {
     // ------------------------------------------------------------------ MMA issuer
-    const uint32_t idesc = fp.fp8 ? make_idesc_e4m3(N_PAD) : make_idesc(N_PAD);
+    const uint32_t idesc = kFp8 ? make_idesc_e4m3(N_PAD) : make_idesc(N_PAD);
     int ws_i = 0, hs_i = 0;
     uint32_t wph = 0, hph = 0;
     bool ok = true;
@@ -310,7 +312,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           for (int k = 0; k < 4; ++k) {   // four MMAs of 32 bytes of K each: 16 bf16 or 32 FP8 codes
             const uint64_t da = make_smem_desc(wb + k * 32), db = make_smem_desc(hb + k * 32);
             const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-            if (fp.fp8) umma_e4m3(dcol, da, db, idesc, acc);
+            if constexpr (kFp8) umma_e4m3(dcol, da, db, idesc, acc);
             else umma_bf16(dcol, da, db, idesc, acc);
           }
           umma_commit(smem_u32(&ms.empty_w[ws_i]));
@@ -965,11 +967,11 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   }
 }
 
-template <int N_PAD>
+template <int N_PAD, bool kFp8>
 cudaError_t launch_fused(const CUtensorMap& tmW, const CUtensorMap& tmH, const CallParams& cp, const Workspace& ws,
                          const void* H, const void* wj, const float* w_scale, const FusedParams& fp,
                          const FusedPlan& plan, cudaStream_t st) {
-  auto kern = fused_verify_kernel<N_PAD>;
+  auto kern = fused_verify_kernel<N_PAD, kFp8>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
   if (e != cudaSuccess) return e;
   const __nv_bfloat16* Hp = (const __nv_bfloat16*)H;
@@ -1036,12 +1038,18 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
   fp.off_w = (fp.off_w + 1023u) & ~1023u;
   cudaError_t e;
   switch (plan.n_pad) {
-    case 16: e = launch_fused<16>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 32: e = launch_fused<32>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 48: e = launch_fused<48>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 64: e = launch_fused<64>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 80: e = launch_fused<80>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 96: e = launch_fused<96>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 16: e = fp.fp8 ? launch_fused<16, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
+                       : launch_fused<16, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 32: e = fp.fp8 ? launch_fused<32, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
+                       : launch_fused<32, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 48: e = fp.fp8 ? launch_fused<48, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
+                       : launch_fused<48, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 64: e = fp.fp8 ? launch_fused<64, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
+                       : launch_fused<64, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 80: e = fp.fp8 ? launch_fused<80, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
+                       : launch_fused<80, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 96: e = fp.fp8 ? launch_fused<96, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
+                       : launch_fused<96, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
     default: e = cudaErrorInvalidValue; break;
   }
   *err = e;

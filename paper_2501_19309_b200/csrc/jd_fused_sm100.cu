@@ -742,7 +742,8 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           float dv[4][8], lg[4][8];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            const int b = min(b0 + q, cp.B - 1);
+            if (b0 + q >= cp.B) continue;   // uniform over the CTA: no work for sequences that do not exist
+            const int b = b0 + q;
             const int row = ms.sel_row[b], kind = ms.sel_kind[b];
             const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;   // read only when kind == 0
 #pragma unroll
@@ -753,13 +754,15 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           }
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            const int b = min(b0 + q, cp.B - 1);
+            if (b0 + q >= cp.B) continue;   // uniform over the CTA: no work for sequences that do not exist
+            const int b = b0 + q;
             const int col = fp.sample_only ? b : ms.sel_row[b];   // TMEM column of this sequence's selected row
             load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], &ms.swt[0][0], lg[q]);
           }
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
-            const int b = min(b0 + q, cp.B - 1);
+            if (b0 + q >= cp.B) continue;   // uniform over the CTA: no work for sequences that do not exist
+            const int b = b0 + q;
             const int kind = ms.sel_kind[b];
             const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
 #pragma unroll

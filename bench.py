@@ -126,6 +126,7 @@ def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, 
                 "algorithmic_bytes": bytes_alg, "kernel_ms": kernel_ms}
     ach = flops / (kernel_ms * 1e-3) / 1e12
     return {"bound": "tensor", "achieved": ach, "peak": tf_peak, "unit": "TFLOP/s", "frac": ach / tf_peak,
+            "frac_of_sustained_peak": ach / peaks["bf16_tflops_sustained"],
             "traffic": traffic, "peak_source": which, "algorithmic_flops": flops, "kernel_ms": kernel_ms}
 
 

@@ -185,6 +185,13 @@ jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* args, void* cu
  * *out = JD_OK, JD_ERR_TIMEOUT or JD_ERR_BAD_TOKEN. */
 jd_status_t jd_last_device_status(jd_handle_t h, int* out);
 
+/* Test helper for the failure path: launches a two-CTA kernel whose barrier wait can never be
+ * satisfied and gives up after `spin_limit` polls (1 .. 2^20, about 40 ns each). No memory is
+ * touched beyond the handle's status word; afterwards jd_last_device_status reports
+ * JD_ERR_TIMEOUT and the handle stays usable. Every wait inside the real kernels is bounded the
+ * same way (limit 2^22). */
+jd_status_t jd_selftest_timeout(jd_handle_t h, uint32_t spin_limit, void* cuda_stream);
+
 /* Variant the last jd_verify on this handle ran (jd_variant_t), 0 before the first call, and
  * the number of kernels it launched. Either pointer may be NULL. */
 jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launches);

@@ -414,6 +414,17 @@ jd_status_t jd_last_device_status(jd_handle_t h, int* out) {
   return JD_OK;
 }
 
+jd_status_t jd_selftest_timeout(jd_handle_t h, uint32_t spin_limit, void* cuda_stream) {
+  if (!h || spin_limit < 1 || spin_limit > (1u << 20)) return JD_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return JD_ERR_CUDA;
+  if (cudaMemsetAsync(h->ws.status, 0, 512, st) != cudaSuccess) return JD_ERR_CUDA;
+  launch_timeout_probe(h->ws, spin_limit, st);
+  if (cudaGetLastError() != cudaSuccess) return JD_ERR_CUDA;
+  h->last_stream = st;
+  return JD_OK;
+}
+
 jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launches) {
   if (!h) return JD_ERR_INVALID_ARG;
   if (variant) *variant = h->last_variant;

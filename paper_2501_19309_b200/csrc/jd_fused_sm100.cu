@@ -984,7 +984,21 @@ cudaError_t launch_fused(const CUtensorMap& tmW, const CUtensorMap& tmH, const C
                                      st);
 }
 
+// Self-test of the bounded wait: two CTAs arrive at a barrier that expects three, so the wait can
+// only end by running out of its (short) limit; each records JD_ERR_TIMEOUT and returns.
+__global__ void timeout_probe_kernel(Workspace ws, unsigned limit) {
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    if (!grid_arrive_and_wait(ws.barrier + 7, gridDim.x + 1, &abort_flag, limit)) set_status(ws.status, JD_ERR_TIMEOUT);
+  }
+}
+
 }  // namespace
+
+void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st) {
+  timeout_probe_kernel<<<2, 32, 0, st>>>(ws, limit);
+}
 
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan) {
   const bool fp8 = dtype == JD_DTYPE_FP8_E4M3;

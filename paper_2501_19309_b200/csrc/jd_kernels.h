@@ -31,6 +31,7 @@ struct FusedPlan {
   size_t smem_bytes;  // dynamic shared memory of the launch
   int stages;         // W ring depth
 };
+void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st);
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan);
 // Returns the number of kernels launched, or -1 with *err set.
 int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,

@@ -125,10 +125,11 @@ __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" :::
 
 // Grid barrier on a global counter; thread 0 of the epilogue group calls it. Cooperative launch
 // guarantees co-residency; the spin is bounded all the same.
-__device__ __forceinline__ bool grid_arrive_and_wait(unsigned* counter, unsigned expected, volatile int* abort_flag) {
+__device__ __forceinline__ bool grid_arrive_and_wait(unsigned* counter, unsigned expected, volatile int* abort_flag,
+                                                     unsigned limit = kSpinLimit) {
   __threadfence();
   atomicAdd(counter, 1u);
-  for (unsigned it = 0; it < kSpinLimit; ++it) {
+  for (unsigned it = 0; it < limit; ++it) {
     unsigned v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
     if (v >= expected) return true;

@@ -33,7 +33,7 @@ VARIANTS = {"auto": JD_VARIANT_AUTO, "simt": JD_VARIANT_SIMT, "fused": JD_VARIAN
 
 EXPORTS = ["jd_version", "jd_status_string", "jd_workspace_bytes", "jd_create", "jd_destroy", "jd_set_head",
            "jd_verify", "jd_verify_host", "jd_last_device_status", "jd_last_launch_info", "jd_philox_uniforms",
-           "jd_verify_static", "jd_set_head_fp8"]
+           "jd_verify_static", "jd_set_head_fp8", "jd_selftest_timeout"]
 
 
 class jd_config_t(C.Structure):
@@ -77,6 +77,7 @@ def load():
     lib.jd_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(jd_config_t)]
     lib.jd_destroy.argtypes = [C.c_void_p]
     lib.jd_set_head.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
+    lib.jd_selftest_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
     lib.jd_set_head_fp8.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
     lib.jd_verify.argtypes = [C.c_void_p, C.POINTER(jd_verify_args_t), C.c_void_p]
     lib.jd_verify_host.argtypes = [C.c_void_p, C.POINTER(jd_verify_args_t), C.c_void_p]
@@ -133,6 +134,10 @@ def jd_verify(h, args: jd_verify_args_t, stream_ptr: int = 0) -> int:
 
 def jd_verify_host(h, args: jd_verify_args_t, stream_ptr: int = 0) -> int:
     return load().jd_verify_host(h, C.byref(args), C.c_void_p(stream_ptr))
+
+
+def jd_selftest_timeout(h, spin_limit: int, stream_ptr: int = 0) -> int:
+    return load().jd_selftest_timeout(h, C.c_uint32(spin_limit), C.c_void_p(stream_ptr))
 
 
 def jd_last_device_status(h) -> int:

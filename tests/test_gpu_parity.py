@@ -398,3 +398,62 @@ def test_fp8_fused_matches_fp8_simt_and_row_codes_match_checker():
     args, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, variant="batched")
     assert jd.jd_verify(ver.h, args) == jd.JD_ERR_UNSUPPORTED
     ver.close()
+
+
+# ------------------------------------------------------------------ failure path and edge shapes
+def test_bounded_wait_reports_timeout_and_handle_stays_usable():
+    from paper_2501_19309_b200 import jd
+    wl = I.CONFIGS[1].scaled("small", d=128, V=3000, B=2, M=4)
+    inp = I.make_inputs(wl, 1)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    assert jd.jd_selftest_timeout(ver.h, 2000) == jd.JD_OK        # a wait nothing can satisfy, ~0.1 ms
+    assert ver.device_status() == jd.JD_ERR_TIMEOUT
+    assert jd.jd_selftest_timeout(ver.h, 0) == jd.JD_ERR_INVALID_ARG
+    got = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "judge_or_standard"))
+    assert ver.device_status() == jd.JD_OK                        # the next call starts clean
+    T.compare(got, T.run_oracle(inp, "judge_or_standard", seed=0), "judge_or_standard", wl.M)
+    ver.close()
+
+
+@pytest.mark.parametrize("B,M,d,V", [(1, 95, 64, 2000), (48, 1, 64, 5000), (1, 1, 64, 2), (2, 2, 64, 129)])
+def test_extreme_shapes(B, M, d, V):
+    wl = I.CONFIGS[2].scaled("edge-%d-%d-%d-%d" % (B, M, d, V), B=B, M=M, d=d, V=V)
+    seqs = None if B <= 4 else [0, B - 1]
+    for variant in ("fused", "simt"):
+        run_case(wl, 17, variant=variant, modes=("judge_or_standard",), seeds=[0], sequences=seqs,
+                 expect_variant=variant)
+
+
+def test_boundary_tokens_and_forced_outcomes():
+    import torch
+    wl = I.CONFIGS[1].scaled("bt", B=3, M=5, d=128, V=128 * 9)
+    inp = I.make_inputs(wl, 19)
+    inp.draft_tokens[0, :] = [0, wl.V - 1, 127, 128, wl.V - 129]           # tile edges and vocabulary ends
+    inp.draft_tokens[1, :] = inp.draft_tokens[1, 0]                         # the same token in every slot
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    for variant in ("fused", "simt"):
+        for tau, mode in ((0.0, "judge"), (1.0, "judge"), (0.5, "standard")):   # all accepted / all rejected / mixed
+            got = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], tau, 2, mode, variant=variant))
+            T.compare(got, T.run_oracle(inp, mode, seed=2, tau=tau), mode, wl.M)
+            if mode == "judge":
+                assert (got["accept_len"] == (wl.M if tau == 0.0 else 0)).all()
+    ver.close()
+
+
+def test_host_entry_point_with_batched_and_fp8_handles():
+    import torch
+    for dtype, B, M in (("bf16", 8, 16), ("fp8", 2, 6)):
+        wl = I.CONFIGS[2].scaled("host-" + dtype, B=B, M=M, d=128, V=30000, dtype=dtype)
+        inp = I.make_inputs(wl, 23)
+        dev = T.upload(inp)
+        ver = T.make_verifier(inp, dev)
+        want = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 5, "judge_or_standard"))
+        hH = torch.from_numpy(inp.H).view(torch.bfloat16).pin_memory()
+        hx = torch.from_numpy(inp.draft_tokens).pin_memory()
+        hdl = torch.from_numpy(inp.draft_logits).pin_memory()
+        got = {k: v.numpy().copy() for k, v in ver.verify_host(hH, hx, hdl, 0.5, 5, "judge_or_standard").items()}
+        for k in want:
+            assert np.array_equal(want[k], got[k]), (dtype, k)
+        ver.close()

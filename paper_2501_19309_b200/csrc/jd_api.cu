@@ -242,7 +242,8 @@ jd_status_t jd_set_head_fp8(jd_handle_t h, const void* W8, const float* w_scale,
   h->head_set = true;
   h->tm_w_ok = false;
   if (h->cfg.d % 128 == 0)
-    h->tm_w_ok = make_tensor_map(&h->tm_w, W8, (uint64_t)h->cfg.V, (uint64_t)h->cfg.d, 128, true);
+    h->tm_w_ok = make_tensor_map(&h->tm_w, W8, (uint64_t)h->cfg.V, (uint64_t)h->cfg.d, 128, true) &&
+                 make_tensor_map(&h->tm_w256, W8, (uint64_t)h->cfg.V, (uint64_t)h->cfg.d, 256, true);
   return JD_OK;
 }
 
@@ -285,7 +286,7 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   FusedPlan plan;
   const bool fused_ok = h->tm_w_ok && fused_supported(c.dtype, R, c.d, c.V, h->num_sms, &plan);
   const bool fp8 = c.dtype == JD_DTYPE_FP8_E4M3;
-  const bool batched_ok = !fp8 && h->tm_w_ok && batched_supported(c.dtype, a->B, c.d, c.V, h->num_sms);
+  const bool batched_ok = h->tm_w_ok && batched_supported(c.dtype, a->B, c.d, c.V, h->num_sms);
   int variant = a->variant;
   if (variant == JD_VARIANT_AUTO) {
     if (a->logits_debug) variant = JD_VARIANT_SIMT;
@@ -319,11 +320,12 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
     FusedPlan plan2;   // second pass: B rows through the fused kernel
     if (!fused_supported(c.dtype, a->B, c.d, c.V, h->num_sms, &plan2)) return JD_ERR_UNSUPPORTED;
     CUtensorMap tm_h, tm_hsel;
-    if (!make_tensor_map(&tm_h, a->H, (uint64_t)R, (uint64_t)c.d, 128) ||
-        !make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)a->B, (uint64_t)c.d, (uint32_t)plan2.n_pad))
+    if (!make_tensor_map(&tm_h, fp8 ? (const void*)h->ws.h8 : a->H, (uint64_t)R, (uint64_t)c.d, 128, fp8) ||
+        !make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)a->B, (uint64_t)c.d, (uint32_t)plan2.n_pad, fp8))
       return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
-    const int n = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, a->H, h->w_judge, h->num_sms, st, h->side, &err);
+    const int n = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, a->H, h->w_judge, h->num_sms, st, h->side,
+                              &err, fp8 ? h->w_scale : nullptr);
     if (n < 0) return JD_ERR_CUDA;
     launches += n;
   } else {

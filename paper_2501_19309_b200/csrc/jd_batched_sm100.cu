@@ -20,18 +20,20 @@ namespace {
 constexpr int kBThreads = 192;
 constexpr int kTileM = 128;   // rows per tile
 constexpr int kTileN = 256;   // vocabulary entries per tile
-constexpr int kTileK = 64;    // bf16 per k-step (one 128-byte swizzle row)
+constexpr int kTileK = 64;    // bf16 per k-step (one 128-byte swizzle row); E4M3 codes: 128 per k-step
 constexpr int kAStage = kTileM * 128;   // 16 KB
 constexpr int kBStage = kTileN * 128;   // 32 KB
 constexpr int kBStages = 4;
-constexpr int kBMisc = 1024;
+constexpr int kBMisc = 3072;
 
 struct BMisc {
   uint64_t full[kBStages], empty[kBStages];
   uint64_t tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort_flag;
+  float wsc[2][kTileN];   // E4M3 head: weight scales of the tile in each accumulator buffer
 };
+static_assert(sizeof(BMisc) <= kBMisc, "BMisc outgrew its shared-memory slot");
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   uint32_t r[32];
@@ -50,14 +52,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// kFp8: W and the quantised rows of H (ws.h8) are E4M3 codes, multiplied by kind::f8f6f4 MMAs (K = 32
+//       codes per instruction, 128 per k-step); the epilogue applies the scale of the vocabulary row
+//       and of the H row to every accumulator. A template parameter, so that the MMA loop of one
+//       instantiation names one instruction kind only.
 // kCount == false: softmax statistics + gather (first pass).
 // kCount == true : top-K rule, after the fold: the same GEMM again (bit-identical logits), the
 //                  epilogue counts the entries that rank above the drafted token and records the
 //                  lowest token id equal to the folded row maximum.
-template <bool kCount>
+template <bool kCount, bool kFp8>
 __global__ void __launch_bounds__(kBThreads, 1)
 gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, CallParams cp,
-                  Workspace ws, int R, int np) {
+                  Workspace ws, int R, int np, const float* __restrict__ w_scale) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   BMisc& ms = *reinterpret_cast<BMisc*>(smem);
@@ -67,7 +73,8 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x;
   volatile int* abort_flag = &ms.abort_flag;
-  const int num_kb = cp.d / kTileK;
+  constexpr int kStepElems = kFp8 ? 2 * kTileK : kTileK;   // elements per 128-byte k-step
+  const int num_kb = cp.d / kStepElems;
   const int row_blocks = (R + kTileM - 1) / kTileM;
   const int voc_blocks = (cp.V + kTileN - 1) / kTileN;
   const int num_tiles = row_blocks * voc_blocks;
@@ -101,14 +108,14 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         ok = mbar_wait(smem_u32(&ms.empty[s]), ph ^ 1u, abort_flag);
         if (!ok) break;
         mbar_expect_tx(smem_u32(&ms.full[s]), kAStage + kBStage);
-        tma_load_2d(sA + s * kAStage, &tmH, smem_u32(&ms.full[s]), kb * kTileK, rb * kTileM, pol_h);
-        tma_load_2d(sB + s * kBStage, &tmW, smem_u32(&ms.full[s]), kb * kTileK, vb * kTileN, pol_w);
+        tma_load_2d(sA + s * kAStage, &tmH, smem_u32(&ms.full[s]), kb * kStepElems, rb * kTileM, pol_h);
+        tma_load_2d(sB + s * kBStage, &tmW, smem_u32(&ms.full[s]), kb * kStepElems, vb * kTileN, pol_w);
         if (++s == kBStages) { s = 0; ph ^= 1u; }
       }
     }
     if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
   } else if (warp == 5 && lane == 0) {
-    const uint32_t idesc = make_idesc(kTileN);
+    const uint32_t idesc = kFp8 ? make_idesc_e4m3(kTileN) : make_idesc(kTileN);
     int s = 0;
     uint32_t ph = 0;
     bool ok = true;
@@ -125,8 +132,11 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         tc_fence_after();
         const uint32_t ab = sA + s * kAStage, bb = sB + s * kBStage;
 #pragma unroll
-        for (int k = 0; k < kTileK / 16; ++k)
-          umma_bf16(dcol, make_smem_desc(ab + k * 32), make_smem_desc(bb + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+        for (int k = 0; k < 4; ++k) {   // 32 bytes of K per instruction: 16 bf16 or 32 codes
+          const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+          if constexpr (kFp8) umma_e4m3(dcol, make_smem_desc(ab + k * 32), make_smem_desc(bb + k * 32), idesc, acc);
+          else umma_bf16(dcol, make_smem_desc(ab + k * 32), make_smem_desc(bb + k * 32), idesc, acc);
+        }
         umma_commit(smem_u32(&ms.empty[s]));
         if (++s == kBStages) { s = 0; ph ^= 1u; }
       }
@@ -151,6 +161,10 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           if (x < 0 || x >= cp.V) { set_status(ws.status, JD_ERR_BAD_TOKEN); x = min(max(x, 0), cp.V - 1); }
         }
       }
+      if (kFp8) {   // the previous reader of this buffer's scales finished two tiles (and two syncs) ago
+        ms.wsc[buf][tid] = v0 + tid < cp.V ? __ldg(w_scale + v0 + tid) : 0.f;
+        ms.wsc[buf][tid + 128] = v0 + tid + 128 < cp.V ? __ldg(w_scale + v0 + tid + 128) : 0.f;
+      }
       if (tid == 0) mbar_wait(smem_u32(&ms.tmem_full[buf]), (uint32_t)(it >> 1) & 1u, abort_flag);
       epi_sync();
       ok = (*abort_flag == 0);
@@ -160,7 +174,8 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       bool have_g = false;
       int above = 0, cand = 0x7F7F7F7F;
       float g_ref = 0.f, rmax = 0.f;
-      const float sc = (cp.norm == JD_NORM_RMS && row < R) ? ws.row_scale[row] : 1.f;
+      float sc = (cp.norm == JD_NORM_RMS && row < R) ? ws.row_scale[row] : 1.f;
+      if (kFp8 && row < R) sc *= ws.h_scale[row];
       if (kCount && row < R) {
         rmax = ws.row_max[row];
         if (x >= 0) g_ref = ws.gath[row];
@@ -169,8 +184,13 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       for (int c0 = 0; c0 < kTileN; c0 += 32) {
         float v[32];
         tmem_ld32(lane_base + (uint32_t)(buf * kTileN + c0), v);
+        if (kFp8) {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) v[k] *= sc;
+          for (int k = 0; k < 32; ++k) v[k] = (v[k] * ms.wsc[buf][c0 + k]) * sc;
+        } else {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) v[k] *= sc;
+        }
         const int nvalid = cp.V - (v0 + c0);   // columns of this chunk that exist (>= 32 except at the tail)
         if (nvalid < 32) {
 #pragma unroll
@@ -235,13 +255,15 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 // matrix, and the selected draft-logit row (where the residual needs it) into a tile-major
 // buffer [vocab tile][sequence][128], so that a CTA of the second pass finds the draft logits of
 // its vocabulary slice for all sequences in one contiguous block.
-__global__ void __launch_bounds__(256) gather_rows_kernel(CallParams cp, Workspace ws, const __nv_bfloat16* __restrict__ H) {
+// `H` is the matrix the second pass multiplies: bf16 rows, or (row_bytes = d) the E4M3 codes.
+__global__ void __launch_bounds__(256) gather_rows_kernel(CallParams cp, Workspace ws, const uint8_t* __restrict__ H,
+                                                          int row_bytes) {
   const int b = blockIdx.x, part = blockIdx.y, parts = gridDim.y;
   const int row = ws.sel_row[b];
   if (part == 0) {
-    const uint4* src = reinterpret_cast<const uint4*>(H + (size_t)row * cp.d);
-    uint4* dst = reinterpret_cast<uint4*>(ws.h_sel + (size_t)b * cp.d);
-    for (int k = threadIdx.x; k < cp.d / 8; k += blockDim.x) dst[k] = src[k];
+    const uint4* src = reinterpret_cast<const uint4*>(H + (size_t)row * row_bytes);
+    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(ws.h_sel) + (size_t)b * row_bytes);
+    for (int k = threadIdx.x; k < row_bytes / 16; k += blockDim.x) dst[k] = src[k];
   }
   if (ws.sel_kind[b] != 0) return;
   const float* dl = cp.draft_logits + ((size_t)b * cp.M + (row % (cp.M + 1))) * cp.V;
@@ -251,8 +273,14 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(CallParams cp, Workspa
 
 }  // namespace
 
+static int grid_of(int R, int np, int num_sms) {
+  return std::min(num_sms, ((R + kTileM - 1) / kTileM) * np);
+}
+
 bool batched_supported(int dtype, int B, int d, int V, int num_sms) {
-  if (dtype != JD_DTYPE_BF16 || d % kTileK != 0 || d < kTileK) return false;
+  if (dtype == JD_DTYPE_BF16) { if (d % kTileK != 0 || d < kTileK) return false; }
+  else if (dtype == JD_DTYPE_FP8_E4M3) { if (d % (2 * kTileK) != 0 || d < 2 * kTileK) return false; }
+  else return false;
   if (num_sms < 1 || num_sms > kMaxCtas) return false;
   FusedPlan plan;
   return fused_supported(dtype, B, d, V, num_sms, &plan);   // the second pass runs B rows through the fused kernel
@@ -260,22 +288,26 @@ bool batched_supported(int dtype, int B, int d, int V, int num_sms) {
 
 int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
                 const CUtensorMap& tmH, const CUtensorMap& tmHsel, const void* H, const void* w_judge, int num_sms,
-                cudaStream_t st, const SideStream& side, cudaError_t* err) {
+                cudaStream_t st, const SideStream& side, cudaError_t* err, const float* w_scale_fp8) {
+  const bool fp8 = w_scale_fp8 != nullptr;
+  const int dtype = fp8 ? JD_DTYPE_FP8_E4M3 : JD_DTYPE_BF16;
   const int R = cp.B * (cp.M + 1);
   const int np = (cp.V + kTileN - 1) / kTileN;
   const size_t smem = 1024 + kBMisc + (size_t)kBStages * (kAStage + kBStage);
-  *err = cudaFuncSetAttribute(gemm_stats_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (*err == cudaSuccess)
-    *err = cudaFuncSetAttribute(gemm_stats_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (*err != cudaSuccess) return -1;
-  const int row_blocks = (R + kTileM - 1) / kTileM, voc_blocks = np;
-  const int grid = std::min(num_sms, row_blocks * voc_blocks);
+  auto gemm = [&](bool count) {
+    auto kern = fp8 ? (count ? gemm_stats_kernel<true, true> : gemm_stats_kernel<false, true>)
+                    : (count ? gemm_stats_kernel<true, false> : gemm_stats_kernel<false, false>);
+    *err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (*err != cudaSuccess) return false;
+    kern<<<grid_of(R, np, num_sms), kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np, w_scale_fp8);
+    return true;
+  };
   int nq;
   if (side.stream) {
     // The draft statistics (HBM-bound) and the judge dots do not depend on the GEMM (tensor-bound):
     // they run on the handle's side stream next to it and join before the decision.
     if ((*err = cudaEventRecord(side.fork, st)) != cudaSuccess) return -1;
-    gemm_stats_kernel<false><<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+    if (!gemm(false)) return -1;
     if ((*err = cudaStreamWaitEvent(side.stream, side.fork, 0)) != cudaSuccess) return -1;
     nq = launch_q_stats(cp, ws, side.stream);
     launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, side.stream);
@@ -284,19 +316,20 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
   } else {
     nq = launch_q_stats(cp, ws, st);
     launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, st);
-    gemm_stats_kernel<false><<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+    if (!gemm(false)) return -1;
   }
   launch_fold(cp, ws, np, nq, st);
   if (cp.rule == JD_RULE_TOPK) {   // second GEMM pass for ranks and argmax; no token draw
-    gemm_stats_kernel<true><<<grid, kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np);
+    if (!gemm(true)) return -1;
     launch_decide(cp, ws, st);
     return 6;
   }
   launch_decide(cp, ws, st);
-  gather_rows_kernel<<<dim3(cp.B, 8), 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H);
+  // second pass operand: the bf16 rows, or their E4M3 codes (one byte per element)
+  gather_rows_kernel<<<dim3(cp.B, 8), 256, 0, st>>>(cp, ws, fp8 ? ws.h8 : (const uint8_t*)H, fp8 ? cp.d : cp.d * 2);
   FusedPlan plan;
-  if (!fused_supported(JD_DTYPE_BF16, cp.B, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }
-  const int n = run_fused(cp, ws, tmW128, tmHsel, ws.h_sel, w_judge, plan, st, err, /*sample_only=*/true);
+  if (!fused_supported(dtype, cp.B, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }
+  const int n = run_fused(cp, ws, tmW128, tmHsel, ws.h_sel, w_judge, plan, st, err, /*sample_only=*/true, w_scale_fp8);
   if (n < 0) return -1;
   return 6 + n;
 }

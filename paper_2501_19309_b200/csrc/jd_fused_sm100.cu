@@ -231,7 +231,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     ms.x_row[tid] = x;
     float f = 1.f;   // normalisation factor of the row held in TMEM column tid
     if (cp.norm == JD_NORM_RMS && tid < R) f = ws.row_scale[fp.sample_only ? ws.sel_row[tid] : tid];
-    if (fp.fp8 && tid < R) f *= ws.h_scale[tid];
+    if (fp.fp8 && tid < R) f *= ws.h_scale[fp.sample_only ? ws.sel_row[tid] : tid];
     ms.scale[tid] = f;
   }
   if (tid < kVocabTile) {   // per-vocabulary-row scales of an FP8 head, one per tile of this CTA; 1 otherwise

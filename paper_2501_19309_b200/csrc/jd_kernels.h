@@ -40,7 +40,8 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
 
 // Two-pass tensor-core variant for many rows (jd_batched_sm100.cu). tmW256 / tmW128: W with
 // 256- and 128-row boxes; tmH: H with a 128-row box; tmHsel: the handle's [B, d] gather buffer
-// with the fused plan's box. Returns the number of kernels launched, or -1 with *err set.
+// with the fused plan's box. With w_scale_fp8 set, W is E4M3 and tmH / tmHsel describe the
+// quantised rows (ws.h8) and the gather buffer as bytes. Returns the number of kernels launched, or -1 with *err set.
 // Optional second stream of a handle (with the two events that fork to it and join from it).
 struct SideStream {
   cudaStream_t stream;
@@ -49,6 +50,6 @@ struct SideStream {
 bool batched_supported(int dtype, int B, int d, int V, int num_sms);
 int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
                 const CUtensorMap& tmH, const CUtensorMap& tmHsel, const void* H, const void* w_judge, int num_sms,
-                cudaStream_t st, const SideStream& side, cudaError_t* err);
+                cudaStream_t st, const SideStream& side, cudaError_t* err, const float* w_scale_fp8 = nullptr);
 
 }  // namespace jd

@@ -369,6 +369,9 @@ FP8_CASES = [
     ("fused", 4, 16, 128, 40000 + 77),
     ("fused", 1, 25, 512, 128256),
     ("fused", 6, 15, 128, 128256),            # overflow tiles
+    ("batched", 8, 16, 128, 128256),          # two row blocks of the FP8 GEMM, the second mostly padding
+    ("batched", 3, 50, 256, 5000 + 77),       # ragged last vocabulary block, two k-steps
+    ("batched", 64, 16, 128, 20000),          # the serving shape's rows
 ]
 
 
@@ -378,8 +381,9 @@ def test_fp8_head_parity(variant, B, M, d, V):
     rep = run_case(wl, 13, variant=variant, modes=("judge_or_standard", "standard"), seeds=[0, 1],
                    expect_variant=variant, check_logits=(variant == "simt"))
     assert rep.sequences == 4 * B
-    if variant == "fused":
+    if variant != "simt":
         run_case(wl, 13, variant=variant, modes=("standard",), seeds=[0], rule="greedy", rms_eps=1e-5)
+        run_case(wl, 13, variant=variant, modes=("judge_or_standard",), seeds=[0], rule="topk", top_k=7)
 
 
 def test_fp8_fused_matches_fp8_simt_and_row_codes_match_checker():
@@ -392,11 +396,22 @@ def test_fp8_fused_matches_fp8_simt_and_row_codes_match_checker():
     b = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 1, "judge_or_standard", variant="simt"))
     assert np.array_equal(a["accept_len"], b["accept_len"]) and np.array_equal(a["masks"], b["masks"])
     assert np.allclose(a["row_lse"], b["row_lse"], rtol=0, atol=1e-4)
-    # an FP8 handle refuses the bf16 registration call and the batched variant
+    c = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 1, "judge_or_standard", variant="batched"))
+    assert np.array_equal(a["accept_len"], c["accept_len"]) and np.array_equal(a["masks"], c["masks"])
+    assert np.allclose(a["row_lse"], c["row_lse"], rtol=0, atol=1e-4)
+    assert np.allclose(a["p_draft"], c["p_draft"], rtol=1e-4)
+    # an FP8 handle refuses the bf16 registration call
     from paper_2501_19309_b200 import jd
     assert jd.jd_set_head(ver.h, dev["W"].data_ptr(), dev["w"].data_ptr(), 0.0) == jd.JD_ERR_INVALID_ARG
-    args, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, variant="batched")
-    assert jd.jd_verify(ver.h, args) == jd.JD_ERR_UNSUPPORTED
+    ver.close()
+    # the tensor-core variants need whole 128-byte k-steps of codes: d = 192 is refused, not faked
+    wl = I.CONFIGS[2].scaled("fp8y", B=2, M=3, d=192, V=1000, dtype="fp8")
+    inp = I.make_inputs(wl, 2)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    for variant in ("fused", "batched"):
+        args, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, variant=variant)
+        assert jd.jd_verify(ver.h, args) == jd.JD_ERR_UNSUPPORTED
     ver.close()
 
 

@@ -136,7 +136,7 @@ def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, 
 def oracle_step(inp: I.Inputs, seed: int, sequences):
     from oracle import jd_oracle as O
     return O.jd_oracle_verify(inp.W, inp.w_judge, inp.b_judge, inp.H, inp.draft_tokens, inp.draft_logits,
-                              inp.tau, seed, "judge_or_standard", sequences=sequences)
+                              inp.tau, seed, "judge_or_standard", sequences=sequences, w_scale=inp.w_scale)
 
 
 def cpu_threads() -> int:
@@ -280,11 +280,14 @@ def main() -> None:
     ap.add_argument("--config", type=int, default=1, help="workload id of the headline line (1..4)")
     ap.add_argument("--others", default="2,3,4,3f,4f", help="comma list of further workloads summarised in the same "
                     "line; a trailing f = the same shape with an FP8 E4M3 head")
+    ap.add_argument("--fp8", action="store_true", help="headline workload with an FP8 E4M3 head")
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = I.CONFIGS[args.config]
+    if args.fp8:
+        wl = wl.scaled(wl.name + "-fp8", dtype="fp8")
 
     if args.impl == "reference":
         run_reference(args, wl)
@@ -344,7 +347,7 @@ def main() -> None:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
+            "dtype": "fp8" if wl.dtype == "fp8" else "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "B": wl.B, "M": wl.M, "d": wl.d, "V": wl.V, "mode": "judge_or_standard",
                        "variant": VARIANT_NAMES.get(res["variant"], "?"),
                        "l2": "inputs larger than L2: W (%.2f GB) streams from HBM every call" % (wl.V * wl.d * 2 / 1e9),

@@ -109,7 +109,12 @@ def aggregate_value(units_per_rank_step: int, steps: int, world: int, max_second
     return world * units_per_rank_step * steps / max_seconds
 
 
-def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, which: str) -> dict:
+NOMINAL_HBM_GBS = 8000.0      # the "~8 TB/s" the metric's definition quotes
+NOMINAL_BF16_TFLOPS = 2250.0  # dense
+
+
+def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, which: str,
+                stream_gbs: float = None) -> dict:
     if wl.dtype == "fp8":   # one byte per weight + a float per vocabulary row; H read as bf16 once
         bytes_alg = wl.V * wl.d + wl.V * 4 + wl.R * wl.d * 2
     else:
@@ -126,10 +131,13 @@ def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, 
         ach = bytes_alg / (kernel_ms * 1e-3) / 1e9
         return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "peak_source": which,
+                "frac_of_nominal_peak": ach / NOMINAL_HBM_GBS,
+                "read_stream_gbs": stream_gbs, "frac_of_read_stream": ach / stream_gbs if stream_gbs else None,
                 "algorithmic_bytes": bytes_alg, "kernel_ms": kernel_ms}
     ach = flops / (kernel_ms * 1e-3) / 1e12
     return {"bound": "tensor", "achieved": ach, "peak": tf_peak, "unit": "TFLOP/s", "frac": ach / tf_peak,
             "frac_of_sustained_peak": ach / tf_sustained,
+            "frac_of_nominal_peak": ach / (NOMINAL_BF16_TFLOPS * (2 if wl.dtype == "fp8" else 1)),
             "traffic": traffic, "peak_source": which, "algorithmic_flops": flops, "kernel_ms": kernel_ms}
 
 
@@ -239,7 +247,23 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     per = [evs[i].elapsed_time(evs[i + 1]) for i in range(Kp)]
     clocks = sampler.stop() if sampler else None
     assert ver.device_status() == jd.JD_OK
-    accepted = out["accept_len"].cpu().numpy()
+    # tokens a call emits (accepted prefix + the drawn token), averaged over the verify seeds in use
+    accepted = []
+    for i in range(8):
+        step(i)
+        accepted.append(out["accept_len"].cpu().numpy().astype(np.float64))
+    accepted = np.stack(accepted)
+
+    # read-only streaming ceiling of this device: the library's probe over the same W
+    sink = torch.zeros(1, dtype=torch.int32, device=device)
+    w_bytes = W.numel() * W.element_size()
+    pevs = [torch.cuda.Event(enable_timing=True) for _ in range(8)]
+    pevs[0].record(stream)
+    for i in range(7):
+        jd.jd_stream_read_probe(W.data_ptr(), w_bytes, sink.data_ptr(), stream.cuda_stream)
+        pevs[i + 1].record(stream)
+    torch.cuda.synchronize(device)
+    stream_gbs = w_bytes / (statistics.median(pevs[i].elapsed_time(pevs[i + 1]) for i in range(2, 7)) * 1e-3) / 1e9
 
     # end to end: pinned host buffers in, outputs back, every step
     hH = torch.from_numpy(inp.H).view(torch.bfloat16).pin_memory()
@@ -265,7 +289,8 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     ver.close()
     res = dict(total_ms=total_ms, median_ms=statistics.median(per), min_ms=min(per), mean_ms=total_ms / K,
                variant=variant, launches=launches, clocks=clocks, e2e_s=e2e_s, e2e_steps=Ke, h2d=h2d, d2h=d2h,
-               mean_accept=float(accepted.mean()), inp=inp)
+               mean_accept=float(accepted.mean()), emitted_per_call=float((accepted + 1).sum(axis=1).mean()),
+               stream_gbs=stream_gbs, inp=inp)
     del W, H, dl
     torch.cuda.empty_cache()
     return res
@@ -335,9 +360,11 @@ def main() -> None:
                 "B": owl.B, "M": owl.M, "d": owl.d, "V": owl.V, "ms_per_step": r["mean_ms"],
                 "median_ms": r["median_ms"], "value": owl.B * owl.M / (r["mean_ms"] * 1e-3), "unit": UNIT,
                 "variant": VARIANT_NAMES.get(r["variant"], "?"), "kernel_launches_per_step": r["launches"],
-                "steps": small.steps, "mean_accept_len": r["mean_accept"],
+                "steps": small.steps, "mean_accept_len": r["mean_accept"], "best_ms": r["min_ms"],
+                "emitted_tokens_per_s": r["emitted_per_call"] / (r["mean_ms"] * 1e-3),
                 "e2e_value": owl.B * owl.M * r["e2e_steps"] / r["e2e_s"],
-                "roofline": roofline_of(owl, peaks, r["mean_ms"], sustained=r["mean_ms"] * small.steps > 1000, which=which)}
+                "roofline": roofline_of(owl, peaks, r["mean_ms"], sustained=r["mean_ms"] * small.steps > 1000, which=which,
+                                        stream_gbs=r["stream_gbs"])}
 
     if rank == 0:
         cpu = None
@@ -355,11 +382,14 @@ def main() -> None:
                        "mean_accept_len": res["mean_accept"]},
             "calls_per_s": world * K / (total_ms * 1e-3),
             "median_ms_per_step": res["median_ms"],
+            "best_ms_per_step": res["min_ms"],
+            "emitted_tokens_per_s": world * res["emitted_per_call"] * K / (total_ms * 1e-3),
             "clocks": res["clocks"],
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": res["h2d"],
                     "d2h_bytes_per_step": res["d2h"], "steps": res["e2e_steps"]},
             "gpu_launches": res["launches"] * K,
-            "roofline": roofline_of(wl, peaks, res["mean_ms"], sustained=total_ms > 1000, which=which),
+            "roofline": roofline_of(wl, peaks, res["mean_ms"], sustained=total_ms > 1000, which=which,
+                                    stream_gbs=res["stream_gbs"]),
             "cpu_baseline": cpu,
             "other_workloads": others,
         }

@@ -196,6 +196,13 @@ jd_status_t jd_selftest_timeout(jd_handle_t h, uint32_t spin_limit, void* cuda_s
  * the number of kernels it launched. Either pointer may be NULL. */
 jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launches);
 
+/* Measurement aid (the paper has no counterpart): reads the first bytes/16*16 bytes at `data`
+ * (device pointer, 16-byte aligned) exactly once with streaming loads and XORs all 32-bit words
+ * read into *out (device pointer, one word, which the caller zeroes beforehand). The call's
+ * device time over the LM head is the read-only streaming ceiling a verification call that must
+ * fetch W once can approach. Asynchronous on the stream; uses the current device. */
+jd_status_t jd_stream_read_probe(const void* data, size_t bytes, uint32_t* out, void* cuda_stream);
+
 /* Test helper: fills out[i] = Philox uniform for (seed, b[i], slot[i], stream[i]), i < n, with
  * the device generator; device pointers. Used to compare the generator bit for bit with an
  * independent host implementation. */

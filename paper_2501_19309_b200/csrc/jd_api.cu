@@ -427,6 +427,16 @@ jd_status_t jd_selftest_timeout(jd_handle_t h, uint32_t spin_limit, void* cuda_s
   return JD_OK;
 }
 
+jd_status_t jd_stream_read_probe(const void* data, size_t bytes, uint32_t* out, void* cuda_stream) {
+  if (!data || !out || bytes < 16 || !aligned16(data)) return JD_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    return JD_ERR_CUDA;
+  launch_stream_read(data, bytes, out, sms, (cudaStream_t)cuda_stream);
+  return cudaGetLastError() == cudaSuccess ? JD_OK : JD_ERR_CUDA;
+}
+
 jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launches) {
   if (!h) return JD_ERR_INVALID_ARG;
   if (variant) *variant = h->last_variant;

@@ -18,6 +18,7 @@ void launch_row_scale(const CallParams& cp, const Workspace& ws, const void* H, 
 void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st);
 void launch_decide(const CallParams& cp, const Workspace& ws, cudaStream_t st);
 void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream_t st);
+void launch_stream_read(const void* p, size_t bytes, uint32_t* out, int num_sms, cudaStream_t st);
 void launch_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot, const int32_t* stream, int n,
                             float* out, cudaStream_t st);
 

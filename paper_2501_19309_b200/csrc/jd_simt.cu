@@ -392,6 +392,29 @@ __global__ void philox_uniforms_kernel(uint64_t seed, const int32_t* b, const in
   if (i < n) out[i] = philox_uniform(seed, b[i], slot[i], stream[i]);
 }
 
+// Measurement aid: reads `n16` 16-byte words once with streaming loads and folds them into one
+// word per block, so that nothing of the read can be dropped. The time of this kernel over W is
+// the ceiling any kernel that must stream W once can reach on the device at hand.
+__global__ void __launch_bounds__(512) stream_read_kernel(const uint4* __restrict__ p, size_t n16, uint32_t* out) {
+  uint32_t acc = 0;
+  const size_t stride = (size_t)gridDim.x * blockDim.x * 4;
+  size_t i = (size_t)blockIdx.x * blockDim.x * 4 + threadIdx.x;
+  for (; i + 3 * (size_t)blockDim.x < n16; i += stride) {   // four independent loads in flight per thread
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = __ldcs(p + i + (size_t)u * blockDim.x);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+  }
+  for (; i < n16; i += blockDim.x) {   // ragged end of this block's last group
+    const uint4 v = __ldcs(p + i);
+    acc ^= v.x ^ v.y ^ v.z ^ v.w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0 && acc != 0) atomicXor(out, acc);
+}
+
 // -----------------------------------------------------------------------------------------
 // host-side launchers
 // -----------------------------------------------------------------------------------------
@@ -466,6 +489,10 @@ int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const flo
   logits(1, nullptr);
   launch_locate(cp, ws, np, st);
   return 7;
+}
+
+void launch_stream_read(const void* p, size_t bytes, uint32_t* out, int num_sms, cudaStream_t st) {
+  stream_read_kernel<<<num_sms * 4, 512, 0, st>>>((const uint4*)p, bytes / 16, out);
 }
 
 void launch_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot, const int32_t* stream, int n,

@@ -33,7 +33,7 @@ VARIANTS = {"auto": JD_VARIANT_AUTO, "simt": JD_VARIANT_SIMT, "fused": JD_VARIAN
 
 EXPORTS = ["jd_version", "jd_status_string", "jd_workspace_bytes", "jd_create", "jd_destroy", "jd_set_head",
            "jd_verify", "jd_verify_host", "jd_last_device_status", "jd_last_launch_info", "jd_philox_uniforms",
-           "jd_verify_static", "jd_set_head_fp8", "jd_selftest_timeout"]
+           "jd_verify_static", "jd_set_head_fp8", "jd_selftest_timeout", "jd_stream_read_probe"]
 
 
 class jd_config_t(C.Structure):
@@ -85,6 +85,7 @@ def load():
     lib.jd_last_launch_info.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
     lib.jd_philox_uniforms.argtypes = [C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
                                        C.c_void_p]
+    lib.jd_stream_read_probe.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.jd_verify_static.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_float,
                                      C.POINTER(jd_verify_args_t), C.c_void_p, C.c_void_p]
     for name in EXPORTS:
@@ -159,6 +160,12 @@ def jd_philox_uniforms(seed: int, b_ptr: int, slot_ptr: int, stream_idx_ptr: int
     return load().jd_philox_uniforms(C.c_uint64(seed), C.c_void_p(b_ptr), C.c_void_p(slot_ptr),
                                      C.c_void_p(stream_idx_ptr), C.c_int32(n), C.c_void_p(out_ptr),
                                      C.c_void_p(stream_ptr))
+
+
+def jd_stream_read_probe(data_ptr: int, nbytes: int, out_ptr: int, stream_ptr: int = 0) -> int:
+    """Reads nbytes at data_ptr once and XORs every 32-bit word into the word at out_ptr; see jd.h."""
+    return load().jd_stream_read_probe(C.c_void_p(data_ptr), C.c_size_t(nbytes), C.c_void_p(out_ptr),
+                                       C.c_void_p(stream_ptr))
 
 
 def jd_verify_static(d: int, V: int, W_ptr: int, w_judge_ptr: int, b_judge: float, args: jd_verify_args_t,

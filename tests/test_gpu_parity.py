@@ -472,3 +472,19 @@ def test_host_entry_point_with_batched_and_fp8_handles():
         for k in want:
             assert np.array_equal(want[k], got[k]), (dtype, k)
         ver.close()
+
+
+def test_stream_read_probe_reads_every_word_once():
+    import torch
+    from paper_2501_19309_b200 import jd
+    rng = np.random.default_rng(5)
+    for nwords in (4, 4 * 2048 * 4 * 148 + 4 * 37, 12345 * 4 + 3):     # one 16-byte word; ragged groups; 3 words ignored
+        host = rng.integers(0, 2 ** 32, size=nwords, dtype=np.uint32)
+        dev = torch.from_numpy(host.view(np.int32)).cuda()
+        sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+        assert jd.jd_stream_read_probe(dev.data_ptr(), nwords * 4, sink.data_ptr()) == jd.JD_OK
+        torch.cuda.synchronize()
+        want = np.bitwise_xor.reduce(host[: nwords // 4 * 4])
+        assert np.uint32(sink.cpu().numpy().view(np.uint32)[0]) == want
+    assert jd.jd_stream_read_probe(0, 64, sink.data_ptr()) == jd.JD_ERR_INVALID_ARG
+    assert jd.jd_stream_read_probe(dev.data_ptr() + 4, 64, sink.data_ptr()) == jd.JD_ERR_INVALID_ARG

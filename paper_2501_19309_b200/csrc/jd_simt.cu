@@ -3,6 +3,8 @@
 // heads, ragged d) and the on-device second opinion the tests compare the fused kernels
 // with. Its stages that do not touch W (draft statistics, judge dot products, decision,
 // token location) are shared with the batched tensor-core variant.
+#include <algorithm>
+
 #include "jd_kernels.h"
 
 namespace jd {
@@ -243,6 +245,64 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(CallParams cp, Works
   }
 }
 
+// The same quantisation for d % 8 == 0: the row is read once, eight bf16 per 16-byte load, kept
+// in registers across the amax reduction, and written as eight codes per store. kVec = loads
+// per thread (blockDim.x * kVec * 8 >= d). Same float32 operations per element as above.
+template <int kVec>
+__global__ void __launch_bounds__(1024) quantize_rows_vec_kernel(CallParams cp, Workspace ws,
+                                                                 const __nv_bfloat16* __restrict__ H) {
+  __shared__ float s_p[32];
+  __shared__ float s_amax;
+  const int row = blockIdx.x, tid = threadIdx.x, nvec = cp.d / 8;
+  const uint4* h = reinterpret_cast<const uint4*>(H + (size_t)row * cp.d);
+  uint4 v[kVec];
+#pragma unroll
+  for (int u = 0; u < kVec; ++u) {
+    const int idx = tid + u * blockDim.x;
+    v[u] = idx < nvec ? __ldg(h + idx) : make_uint4(0u, 0u, 0u, 0u);
+  }
+  float amax = 0.f;
+#pragma unroll
+  for (int u = 0; u < kVec; ++u) {
+    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {   // a bf16 is the upper half of the float with the same value
+      amax = fmaxf(amax, fabsf(__uint_as_float(w[q] << 16)));
+      amax = fmaxf(amax, fabsf(__uint_as_float(w[q] & 0xFFFF0000u)));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if ((tid & 31) == 0) s_p[tid >> 5] = amax;
+  __syncthreads();
+  if (tid == 0) {
+    float t = 0.f;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t = fmaxf(t, s_p[i]);
+    s_amax = t;
+    ws.h_scale[row] = __fdiv_rn(t, 448.f);
+  }
+  __syncthreads();
+  amax = s_amax;
+  const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+  uint2* out = reinterpret_cast<uint2*>(ws.h8 + (size_t)row * cp.d);
+#pragma unroll
+  for (int u = 0; u < kVec; ++u) {
+    const int idx = tid + u * blockDim.x;
+    if (idx >= nvec) continue;
+    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+    uint32_t pair[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float a = __fmul_rn(__uint_as_float(w[q] << 16), inv);           // element 2q
+      const float b = __fmul_rn(__uint_as_float(w[q] & 0xFFFF0000u), inv);   // element 2q + 1
+      unsigned short p;   // upper byte = code of the first operand, lower byte = code of the second
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(p) : "f"(b), "f"(a));
+      pair[q] = p;
+    }
+    out[idx] = make_uint2(pair[0] | (pair[1] << 16), pair[2] | (pair[3] << 16));
+  }
+}
+
 // Row normalisation factors of JD_NORM_RMS: one block per row, 1 / sqrt(mean_k H[row,k]^2 + eps).
 template <typename T>
 __global__ void __launch_bounds__(256) row_scale_kernel(CallParams cp, Workspace ws, const T* __restrict__ H) {
@@ -432,7 +492,17 @@ void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, cons
 }
 
 void launch_quantize_rows(const CallParams& cp, const Workspace& ws, const void* H_bf16, cudaStream_t st) {
-  quantize_rows_kernel<<<cp.B * (cp.M + 1), 256, 0, st>>>(cp, ws, (const __nv_bfloat16*)H_bf16);
+  const int R = cp.B * (cp.M + 1), nvec = cp.d / 8;
+  const __nv_bfloat16* H = (const __nv_bfloat16*)H_bf16;
+  if (cp.d % 8 != 0 || nvec > 4096) {
+    quantize_rows_kernel<<<R, 256, 0, st>>>(cp, ws, H);
+    return;
+  }
+  const int threads = std::min(1024, (nvec + 31) / 32 * 32);
+  const int per = (nvec + threads - 1) / threads;
+  if (per == 1) quantize_rows_vec_kernel<1><<<R, threads, 0, st>>>(cp, ws, H);
+  else if (per == 2) quantize_rows_vec_kernel<2><<<R, threads, 0, st>>>(cp, ws, H);
+  else quantize_rows_vec_kernel<4><<<R, threads, 0, st>>>(cp, ws, H);
 }
 
 void launch_row_scale(const CallParams& cp, const Workspace& ws, const void* H, int dtype, cudaStream_t st) {

@@ -267,6 +267,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(CallParams cp, Workspa
   }
   if (ws.sel_kind[b] != 0) return;
   const float* dl = cp.draft_logits + ((size_t)b * cp.M + (row % (cp.M + 1))) * cp.V;
+#pragma unroll 4
   for (int v = part * 256 + threadIdx.x; v < cp.V; v += parts * 256)
     ws.w_sel[((size_t)(v / kVocabTile) * cp.B + b) * kVocabTile + (v % kVocabTile)] = __ldg(dl + v);
 }
@@ -326,7 +327,7 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
   }
   launch_decide(cp, ws, st);
   // second pass operand: the bf16 rows, or their E4M3 codes (one byte per element)
-  gather_rows_kernel<<<dim3(cp.B, 8), 256, 0, st>>>(cp, ws, fp8 ? ws.h8 : (const uint8_t*)H, fp8 ? cp.d : cp.d * 2);
+  gather_rows_kernel<<<dim3(cp.B, 32), 256, 0, st>>>(cp, ws, fp8 ? ws.h8 : (const uint8_t*)H, fp8 ? cp.d : cp.d * 2);
   FusedPlan plan;
   if (!fused_supported(dtype, cp.B, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }
   const int n = run_fused(cp, ws, tmW128, tmHsel, ws.h_sel, w_judge, plan, st, err, /*sample_only=*/true, w_scale_fp8);

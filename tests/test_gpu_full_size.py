@@ -10,10 +10,12 @@ from paper_2501_19309_b200 import inputs as I
 pytestmark = pytest.mark.gpu
 
 
-def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None, rule="sampling", top_k=1):
+def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None, rule="sampling", top_k=1, fp8=False):
     """cases: list of (mode, tau or None)."""
     from paper_2501_19309_b200 import jd
     wl = I.CONFIGS[cfg]
+    if fp8:
+        wl = wl.scaled(wl.name + "-fp8", dtype="fp8")
     inp = I.make_inputs(wl, data_seed)
     dev = T.upload(inp)
     ver = T.make_verifier(inp, dev)
@@ -95,4 +97,14 @@ def test_cfg1_greedy_and_top5_rules():
 def test_cfg4_greedy_rule_sampled_sequences():
     rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[5, 60], expect_variant="batched",
                        rule="topk", top_k=1)
+    assert rep.sequences == 2
+
+
+def test_cfg3_fp8_head_full_size():
+    rep, _ = full_case(3, 0, [("judge_or_standard", None)], expect_variant="fused", fp8=True)
+    assert rep.sequences == 1
+
+
+def test_cfg4_fp8_head_sampled_sequences():
+    rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[0, 63], expect_variant="batched", fp8=True)
     assert rep.sequences == 2

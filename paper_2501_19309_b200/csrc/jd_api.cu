@@ -35,6 +35,7 @@ struct jd_handle_s {
   float* st_dl;
   void* st_out;            // accept_len | next_token | judge_scores | p_draft | q_draft | row_max | row_lse | masks
   size_t st_out_bytes;
+  void* st_out_host;       // pinned mirror of st_out: the results come back in one copy
 };
 
 namespace {
@@ -227,6 +228,7 @@ jd_status_t jd_destroy(jd_handle_t h) {
   cudaFree(h->st_x);
   cudaFree(h->st_dl);
   cudaFree(h->st_out);
+  if (h->st_out_host) cudaFreeHost(h->st_out_host);
   delete h;
   return JD_OK;
 }
@@ -358,10 +360,12 @@ jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* a, void* cuda_
     if (cudaMalloc(&h->st_H, maxR * c.d * elem_size(c.dtype)) != cudaSuccess ||
         cudaMalloc((void**)&h->st_x, maxBM * 4) != cudaSuccess ||
         cudaMalloc((void**)&h->st_dl, maxBM * (size_t)c.V * 4) != cudaSuccess ||
-        cudaMalloc(&h->st_out, h->st_out_bytes) != cudaSuccess) {
+        cudaMalloc(&h->st_out, h->st_out_bytes) != cudaSuccess ||
+        cudaMallocHost(&h->st_out_host, h->st_out_bytes) != cudaSuccess) {
       cudaGetLastError();
       cudaFree(h->st_H); cudaFree(h->st_x); cudaFree(h->st_dl); cudaFree(h->st_out);
-      h->st_H = nullptr; h->st_x = nullptr; h->st_dl = nullptr; h->st_out = nullptr;
+      if (h->st_out_host) cudaFreeHost(h->st_out_host);
+      h->st_H = nullptr; h->st_x = nullptr; h->st_dl = nullptr; h->st_out = nullptr; h->st_out_host = nullptr;
       return JD_ERR_ALLOC;
     }
   }
@@ -393,16 +397,20 @@ jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* a, void* cuda_
   jd_status_t s = jd_verify(h, &dev, cuda_stream);
   if (s != JD_OK) return s;
 
-  bool ok = cudaMemcpyAsync(a->accept_len, d_acc, B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
-            cudaMemcpyAsync(a->next_token, d_next, B * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
-            cudaMemcpyAsync(a->judge_scores, d_js, BM * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess &&
-            cudaMemcpyAsync(a->p_draft, d_pd, BM * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (ok && a->q_draft) ok = cudaMemcpyAsync(a->q_draft, d_qd, BM * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (ok && a->masks) ok = cudaMemcpyAsync(a->masks, d_mk, BM, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (ok && a->row_max) ok = cudaMemcpyAsync(a->row_max, d_rm, R * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (ok && a->row_lse) ok = cudaMemcpyAsync(a->row_lse, d_rl, R * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (!ok) return JD_ERR_CUDA;
+  // all results in one device-to-host copy (the sections are a few KB), then plain host copies
+  if (cudaMemcpyAsync(h->st_out_host, h->st_out, off, cudaMemcpyDeviceToHost, st) != cudaSuccess) return JD_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return JD_ERR_CUDA;
+  auto back = [&](void* dst, const void* dev_section, size_t bytes) {
+    if (dst) std::memcpy(dst, (const char*)h->st_out_host + ((const char*)dev_section - o), bytes);
+  };
+  back(a->accept_len, d_acc, B * 4);
+  back(a->next_token, d_next, B * 4);
+  back(a->judge_scores, d_js, BM * 4);
+  back(a->p_draft, d_pd, BM * 4);
+  back(a->q_draft, d_qd, BM * 4);
+  back(a->masks, d_mk, BM);
+  back(a->row_max, d_rm, R * 4);
+  back(a->row_lse, d_rl, R * 4);
   return JD_OK;
 }
 

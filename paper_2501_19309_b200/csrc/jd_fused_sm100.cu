@@ -117,7 +117,6 @@ __device__ __forceinline__ void load_chunk2(int i0, int T, int c0, int n_ovf, in
     }
   }
   tmem_wait_ld32(a, b);
-#pragma unroll
   const float w0 = swt[min(i0, 7) * kVocabTile + tid], w1 = swt[min(i0 + 1, 7) * kVocabTile + tid];
 #pragma unroll
   for (int k = 0; k < 16; ++k) {

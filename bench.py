@@ -247,6 +247,30 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
         evs[i + 1].record(stream)
     torch.cuda.synchronize(device)
     per = [evs[i].elapsed_time(evs[i + 1]) for i in range(Kp)]
+    # the same calls replayed from a CUDA graph (eight calls, one per verify seed, per replay)
+    graph_ms = None
+    if not args.no_graph:
+        cap = torch.cuda.Stream(device)
+        cap.wait_stream(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=cap):
+            cs = torch.cuda.current_stream(device).cuda_stream
+            for i in range(8):
+                st = jd.jd_verify(ver.h, a_args[i], cs)
+                if st != jd.JD_OK:
+                    raise jd.JdError(st, "jd_verify (capture)")
+        reps = max(2, K // 8)
+        for _ in range(2):
+            g.replay()
+        torch.cuda.synchronize(device)
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for _ in range(reps):
+            g.replay()
+        g1.record(stream)
+        torch.cuda.synchronize(device)
+        graph_ms = g0.elapsed_time(g1) / (8 * reps)
+        del g
     clocks = sampler.stop() if sampler else None
     assert ver.device_status() == jd.JD_OK
     # tokens a call emits (accepted prefix + the drawn token), averaged over the verify seeds in use
@@ -292,7 +316,7 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     res = dict(total_ms=total_ms, median_ms=statistics.median(per), min_ms=min(per), mean_ms=total_ms / K,
                variant=variant, launches=launches, clocks=clocks, e2e_s=e2e_s, e2e_steps=Ke, h2d=h2d, d2h=d2h,
                mean_accept=float(accepted.mean()), emitted_per_call=float((accepted + 1).sum(axis=1).mean()),
-               stream_gbs=stream_gbs, inp=inp)
+               stream_gbs=stream_gbs, graph_ms=graph_ms, inp=inp)
     del W, H, dl
     torch.cuda.empty_cache()
     return res
@@ -310,6 +334,7 @@ def main() -> None:
     ap.add_argument("--fp8", action="store_true", help="headline workload with an FP8 E4M3 head")
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = I.CONFIGS[args.config]
@@ -363,6 +388,7 @@ def main() -> None:
                 "median_ms": r["median_ms"], "value": owl.B * owl.M / (r["mean_ms"] * 1e-3), "unit": UNIT,
                 "variant": VARIANT_NAMES.get(r["variant"], "?"), "kernel_launches_per_step": r["launches"],
                 "steps": small.steps, "mean_accept_len": r["mean_accept"], "best_ms": r["min_ms"],
+                "graph_replay_ms_per_step": r["graph_ms"],
                 "emitted_tokens_per_s": r["emitted_per_call"] / (r["mean_ms"] * 1e-3),
                 "e2e_value": owl.B * owl.M * r["e2e_steps"] / r["e2e_s"],
                 "roofline": roofline_of(owl, peaks, r["mean_ms"], sustained=r["mean_ms"] * small.steps > 1000, which=which,
@@ -385,6 +411,7 @@ def main() -> None:
             "calls_per_s": world * K / (total_ms * 1e-3),
             "median_ms_per_step": res["median_ms"],
             "best_ms_per_step": res["min_ms"],
+            "graph_replay_ms_per_step": res["graph_ms"],
             "emitted_tokens_per_s": world * res["emitted_per_call"] * K / (total_ms * 1e-3),
             "clocks": res["clocks"],
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": res["h2d"],

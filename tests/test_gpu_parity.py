@@ -488,3 +488,53 @@ def test_stream_read_probe_reads_every_word_once():
         assert np.uint32(sink.cpu().numpy().view(np.uint32)[0]) == want
     assert jd.jd_stream_read_probe(0, 64, sink.data_ptr()) == jd.JD_ERR_INVALID_ARG
     assert jd.jd_stream_read_probe(dev.data_ptr() + 4, 64, sink.data_ptr()) == jd.JD_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------ streams and graphs
+@pytest.mark.parametrize("variant,B,M,d,V", [("fused", 3, 7, 128, 40000), ("batched", 24, 5, 128, 30000),
+                                             ("simt", 2, 4, 96, 3000)])
+def test_call_can_be_captured_in_a_cuda_graph_and_replayed(variant, B, M, d, V):
+    import torch
+    wl = I.CONFIGS[2].scaled("graph-" + variant, B=B, M=M, d=d, V=V)
+    inp = I.make_inputs(wl, 31)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    want = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 3, "judge_or_standard", variant=variant))
+    out = ver.alloc_outputs(B, M)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 3, "judge_or_standard", variant=variant, out=out,
+                   stream=torch.cuda.current_stream())
+    for _ in range(3):
+        for v in out.values():
+            v.zero_()
+        g.replay()
+        got = T.to_numpy(out)
+        for k in want:
+            assert np.array_equal(want[k], got[k]), (variant, k)
+    del g
+    ver.close()
+
+
+def test_two_handles_on_two_streams_do_not_disturb_each_other():
+    import torch
+    cases = []
+    for i, (B, M, V) in enumerate([(4, 16, 50000), (2, 9, 128256)]):
+        wl = I.CONFIGS[2].scaled("two-%d" % i, B=B, M=M, d=128, V=V)
+        inp = I.make_inputs(wl, 40 + i)
+        dev = T.upload(inp)
+        ver = T.make_verifier(inp, dev)
+        want = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 9, "judge_or_standard"))
+        cases.append((inp, dev, ver, want, torch.cuda.Stream(), ver.alloc_outputs(B, M)))
+    torch.cuda.synchronize()
+    for _ in range(5):                      # interleaved, nothing synchronises between the two streams
+        for inp, dev, ver, want, st, out in cases:
+            ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 9, "judge_or_standard", out=out, stream=st)
+    torch.cuda.synchronize()
+    for inp, dev, ver, want, st, out in cases:
+        got = T.to_numpy(out)
+        for k in want:
+            assert np.array_equal(want[k], got[k]), k
+        ver.close()

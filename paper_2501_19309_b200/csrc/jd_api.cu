@@ -319,15 +319,21 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   if (variant == JD_VARIANT_SIMT) {
     launches += run_simt(cp, h->ws, h->W, h->w_scale, h->w_judge, a->H, c.dtype, a->logits_debug, st);
   } else if (variant == JD_VARIANT_BATCHED) {
-    FusedPlan plan2;   // second pass: B rows through the fused kernel
-    if (!fused_supported(c.dtype, a->B, c.d, c.V, h->num_sms, &plan2)) return JD_ERR_UNSUPPORTED;
-    CUtensorMap tm_h, tm_hsel;
+    // second pass: the selected rows go through the fused kernel, a chunk of sequences per launch
+    const int chunk = second_pass_chunk(a->B), tail = a->B % chunk;
+    FusedPlan plan2, plan3;
+    if (!fused_supported(c.dtype, chunk, c.d, c.V, h->num_sms, &plan2)) return JD_ERR_UNSUPPORTED;
+    if (tail && !fused_supported(c.dtype, tail, c.d, c.V, h->num_sms, &plan3)) return JD_ERR_UNSUPPORTED;
+    CUtensorMap tm_h, tm_hsel, tm_hsel_tail;
     if (!make_tensor_map(&tm_h, fp8 ? (const void*)h->ws.h8 : a->H, (uint64_t)R, (uint64_t)c.d, 128, fp8) ||
-        !make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)a->B, (uint64_t)c.d, (uint32_t)plan2.n_pad, fp8))
+        !make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)chunk, (uint64_t)c.d, (uint32_t)plan2.n_pad, fp8))
+      return JD_ERR_CUDA;
+    tm_hsel_tail = tm_hsel;
+    if (tail && !make_tensor_map(&tm_hsel_tail, h->ws.h_sel, (uint64_t)tail, (uint64_t)c.d, (uint32_t)plan3.n_pad, fp8))
       return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
-    const int n = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, a->H, h->w_judge, h->num_sms, st, h->side,
-                              &err, fp8 ? h->w_scale : nullptr);
+    const int n = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, tm_hsel_tail, a->H, h->w_judge, h->num_sms,
+                              st, h->side, &err, fp8 ? h->w_scale : nullptr);
     if (n < 0) return JD_ERR_CUDA;
     launches += n;
   } else {

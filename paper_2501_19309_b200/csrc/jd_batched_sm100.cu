@@ -258,15 +258,18 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 // `H` is the matrix the second pass multiplies: bf16 rows, or (row_bytes = d) the E4M3 codes.
 __global__ void __launch_bounds__(256) gather_rows_kernel(CallParams cp, Workspace ws, const uint8_t* __restrict__ H,
                                                           int row_bytes) {
+  // b counts within the launch's chunk of sequences (ws.sel_* and cp.B are the chunk's views);
+  // the row index is global, and so is the sequence it belongs to
   const int b = blockIdx.x, part = blockIdx.y, parts = gridDim.y;
   const int row = ws.sel_row[b];
+  const int b_global = row / (cp.M + 1);
   if (part == 0) {
     const uint4* src = reinterpret_cast<const uint4*>(H + (size_t)row * row_bytes);
     uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(ws.h_sel) + (size_t)b * row_bytes);
     for (int k = threadIdx.x; k < row_bytes / 16; k += blockDim.x) dst[k] = src[k];
   }
   if (ws.sel_kind[b] != 0) return;
-  const float* dl = cp.draft_logits + ((size_t)b * cp.M + (row % (cp.M + 1))) * cp.V;
+  const float* dl = cp.draft_logits + ((size_t)b_global * cp.M + (row % (cp.M + 1))) * cp.V;
 #pragma unroll 4
   for (int v = part * 256 + threadIdx.x; v < cp.V; v += parts * 256)
     ws.w_sel[((size_t)(v / kVocabTile) * cp.B + b) * kVocabTile + (v % kVocabTile)] = __ldg(dl + v);
@@ -283,13 +286,17 @@ bool batched_supported(int dtype, int B, int d, int V, int num_sms) {
   else if (dtype == JD_DTYPE_FP8_E4M3) { if (d % (2 * kTileK) != 0 || d < 2 * kTileK) return false; }
   else return false;
   if (num_sms < 1 || num_sms > kMaxCtas) return false;
+  // the second pass runs the selected rows through the fused kernel, a chunk of sequences per launch
   FusedPlan plan;
-  return fused_supported(dtype, B, d, V, num_sms, &plan);   // the second pass runs B rows through the fused kernel
+  const int chunk = second_pass_chunk(B);
+  if (!fused_supported(dtype, chunk, d, V, num_sms, &plan)) return false;
+  return B % chunk == 0 || fused_supported(dtype, B % chunk, d, V, num_sms, &plan);
 }
 
 int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
-                const CUtensorMap& tmH, const CUtensorMap& tmHsel, const void* H, const void* w_judge, int num_sms,
-                cudaStream_t st, const SideStream& side, cudaError_t* err, const float* w_scale_fp8) {
+                const CUtensorMap& tmH, const CUtensorMap& tmHsel, const CUtensorMap& tmHselTail, const void* H,
+                const void* w_judge, int num_sms, cudaStream_t st, const SideStream& side, cudaError_t* err,
+                const float* w_scale_fp8) {
   const bool fp8 = w_scale_fp8 != nullptr;
   const int dtype = fp8 ? JD_DTYPE_FP8_E4M3 : JD_DTYPE_BF16;
   const int R = cp.B * (cp.M + 1);
@@ -326,13 +333,27 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
     return 6;
   }
   launch_decide(cp, ws, st);
-  // second pass operand: the bf16 rows, or their E4M3 codes (one byte per element)
-  gather_rows_kernel<<<dim3(cp.B, 32), 256, 0, st>>>(cp, ws, fp8 ? ws.h8 : (const uint8_t*)H, fp8 ? cp.d : cp.d * 2);
-  FusedPlan plan;
-  if (!fused_supported(dtype, cp.B, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }
-  const int n = run_fused(cp, ws, tmW128, tmHsel, ws.h_sel, w_judge, plan, st, err, /*sample_only=*/true, w_scale_fp8);
-  if (n < 0) return -1;
-  return 6 + n;
+  int launches = 5;
+  const int chunk = second_pass_chunk(cp.B);
+  for (int off = 0; off < cp.B; off += chunk) {
+    const int nc = std::min(chunk, cp.B - off);
+    // this chunk's view of the call: sequences off .. off + nc - 1 become 0 .. nc - 1
+    CallParams cc = cp;
+    cc.B = nc;
+    cc.next_token = cp.next_token + off;
+    Workspace wc = ws;
+    wc.sel_row += off; wc.sel_kind += off; wc.sel_lse_p += off; wc.sel_lse_q += off; wc.sel_u += off;
+    if (off > 0 && (*err = cudaMemsetAsync(ws.barrier, 0, 256, st)) != cudaSuccess) return -1;   // grid barriers restart
+    // second pass operand: the bf16 rows, or their E4M3 codes (one byte per element)
+    gather_rows_kernel<<<dim3(nc, 32), 256, 0, st>>>(cc, wc, fp8 ? ws.h8 : (const uint8_t*)H, fp8 ? cp.d : cp.d * 2);
+    FusedPlan plan;
+    if (!fused_supported(dtype, nc, cp.d, cp.V, num_sms, &plan)) { *err = cudaErrorInvalidValue; return -1; }
+    const int n = run_fused(cc, wc, tmW128, nc == chunk ? tmHsel : tmHselTail, ws.h_sel, w_judge, plan, st, err,
+                            /*sample_only=*/true, w_scale_fp8);
+    if (n < 0) return -1;
+    launches += 1 + n;
+  }
+  return launches;
 }
 
 }  // namespace jd

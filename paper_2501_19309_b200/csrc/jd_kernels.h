@@ -48,9 +48,17 @@ struct SideStream {
   cudaStream_t stream;
   cudaEvent_t fork, join;
 };
+// The second pass takes up to 96 sequences in one launch; larger batches go through it 64 at a time
+// (64 selected rows x 7 tiles fill tensor memory exactly), each launch streaming W once more.
+// second_pass_chunk(B) = sequences per launch; tmHsel / tmHselTail describe the gather buffer for a
+// whole chunk and for the ragged last one (ignored when B is a multiple of the chunk).
+constexpr int kSecondPassMax = 96;
+constexpr int kSecondPassChunk = 64;
+inline int second_pass_chunk(int B) { return B <= kSecondPassMax ? B : kSecondPassChunk; }
 bool batched_supported(int dtype, int B, int d, int V, int num_sms);
 int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
-                const CUtensorMap& tmH, const CUtensorMap& tmHsel, const void* H, const void* w_judge, int num_sms,
-                cudaStream_t st, const SideStream& side, cudaError_t* err, const float* w_scale_fp8 = nullptr);
+                const CUtensorMap& tmH, const CUtensorMap& tmHsel, const CUtensorMap& tmHselTail, const void* H,
+                const void* w_judge, int num_sms, cudaStream_t st, const SideStream& side, cudaError_t* err,
+                const float* w_scale_fp8 = nullptr);
 
 }  // namespace jd

@@ -249,6 +249,8 @@ BATCHED_SHAPES = [
     (64, 16, 64, 128256),       # the serving shape's rows (1088) at a narrow d
     (2, 3, 64, 700),            # fewer tiles than CTAs
     (40, 2, 128, 33000),        # many short sequences
+    (130, 3, 64, 9000),         # more sequences than one second-pass launch takes: 64 + 64 + 2
+    (100, 1, 128, 128256),      # 64 + 36 at the full vocabulary
 ]
 
 
@@ -261,8 +263,9 @@ def test_batched_variant_parity(B, M, d, V):
     assert rep.sequences == 4 * (B if seqs is None else len(seqs))
 
 
-def test_batched_matches_simt_on_every_sequence():
-    wl = I.CONFIGS[4].scaled("x", B=48, M=7, d=128, V=20000)
+@pytest.mark.parametrize("B,M", [(48, 7), (150, 3)])
+def test_batched_matches_simt_on_every_sequence(B, M):
+    wl = I.CONFIGS[4].scaled("x", B=B, M=M, d=128, V=20000)
     inp = I.make_inputs(wl, 2)
     dev = T.upload(inp)
     ver = T.make_verifier(inp, dev)
@@ -372,6 +375,7 @@ FP8_CASES = [
     ("batched", 8, 16, 128, 128256),          # two row blocks of the FP8 GEMM, the second mostly padding
     ("batched", 3, 50, 256, 5000 + 77),       # ragged last vocabulary block, two k-steps
     ("batched", 64, 16, 128, 20000),          # the serving shape's rows
+    ("batched", 100, 2, 128, 9000),           # two second-pass launches (64 + 36 sequences)
 ]
 
 

@@ -83,12 +83,14 @@ typedef enum { JD_NORM_NONE = 0, JD_NORM_RMS = 1 } jd_norm_t;
 /* Kernel family used by jd_verify. AUTO picks the fastest one that supports the shape. */
 typedef enum {
   JD_VARIANT_AUTO = 0,
-  JD_VARIANT_SIMT = 1,   /* CUDA-core reference pipeline: any shape, f32 or bf16 */
+  JD_VARIANT_SIMT = 1,   /* CUDA-core reference pipeline: any shape; f32, bf16 or FP8 head */
   JD_VARIANT_FUSED = 2,  /* one persistent tcgen05/TMA kernel, logits parked in tensor memory;
-                            bf16, d % 64 == 0, B*(M+1) <= 96, V small enough for every CTA to
-                            keep its vocabulary tiles on chip (128256 fits on 148 SMs) */
+                            bf16 with d % 64 == 0 or FP8 head with d % 128 == 0, B*(M+1) <= 96, V
+                            small enough for every CTA to keep its vocabulary tiles on chip
+                            (128256 fits on 148 SMs) */
   JD_VARIANT_BATCHED = 3 /* tcgen05 GEMM with fused statistics + second pass over the selected
-                            rows; bf16, d % 64 == 0, any number of rows, B <= 96 */
+                            rows (one launch per 64 sequences beyond 96); same dtypes and d as
+                            the fused variant, any number of rows and sequences */
 } jd_variant_t;
 
 typedef struct {

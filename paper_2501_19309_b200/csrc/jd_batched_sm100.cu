@@ -31,6 +31,7 @@ struct BMisc {
   uint64_t tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort_flag;
+  int go;                 // written by epilogue thread 0 before a sync: 0 once a wait has run out
   float wsc[2][kTileN];   // E4M3 head: weight scales of the tile in each accumulator buffer
 };
 static_assert(sizeof(BMisc) <= kBMisc, "BMisc outgrew its shared-memory slot");
@@ -165,9 +166,12 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         ms.wsc[buf][tid] = v0 + tid < cp.V ? __ldg(w_scale + v0 + tid) : 0.f;
         ms.wsc[buf][tid + 128] = v0 + tid + 128 < cp.V ? __ldg(w_scale + v0 + tid + 128) : 0.f;
       }
-      if (tid == 0) mbar_wait(smem_u32(&ms.tmem_full[buf]), (uint32_t)(it >> 1) & 1u, abort_flag);
+      if (tid == 0) {   // one thread decides for all 128, so that they leave the loop together
+        mbar_wait(smem_u32(&ms.tmem_full[buf]), (uint32_t)(it >> 1) & 1u, abort_flag);
+        ms.go = (*abort_flag == 0);
+      }
       epi_sync();
-      ok = (*abort_flag == 0);
+      ok = ms.go != 0;
       if (!ok) break;
       tc_fence_after();
       float m = -INFINITY, s = 0.f, g = 0.f;

@@ -144,42 +144,6 @@ __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, int 
   for (int u = 0; u < 8; ++u) out[u] = __uint_as_float(raw[u]) * (f * swt[min(i0 + u, 7) * kVocabTile + tid]);
 }
 
-// Reduces 16 per-lane values over the 32 lanes of a warp with 16 shuffles instead of 80: every
-// step halves the number of values a lane keeps. On return lane l holds the reduction of value
-// index reduce16_index(l) (lanes 2j and 2j+1 hold the same one).
-template <bool kMax, typename T>
-__device__ __forceinline__ T warp_reduce16(const T* v, int lane) {
-  auto op = [](T x, T y) { return kMax ? (x > y ? x : y) : x + y; };
-  T a[8], b4[4], c2[2];
-  const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4, h2 = lane & 2;
-#pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const T send = h16 ? v[k] : v[k + 8];
-    const T keep = h16 ? v[k + 8] : v[k];
-    a[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 16));
-  }
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const T send = h8 ? a[k] : a[k + 4];
-    const T keep = h8 ? a[k + 4] : a[k];
-    b4[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 8));
-  }
-#pragma unroll
-  for (int k = 0; k < 2; ++k) {
-    const T send = h4 ? b4[k] : b4[k + 2];
-    const T keep = h4 ? b4[k + 2] : b4[k];
-    c2[k] = op(keep, __shfl_xor_sync(0xffffffffu, send, 4));
-  }
-  const T send = h2 ? c2[0] : c2[1];
-  const T keep = h2 ? c2[1] : c2[0];
-  T d = op(keep, __shfl_xor_sync(0xffffffffu, send, 2));
-  d = op(d, __shfl_xor_sync(0xffffffffu, d, 1));
-  return d;
-}
-__device__ __forceinline__ int reduce16_index(int lane) {
-  return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-}
-
 // kFp8 is a template parameter, not a runtime flag: a kernel whose MMA loop can reach both
 // tcgen05.mma kinds ran its bf16 main loop 40 % slower.
 template <int N_PAD, bool kFp8>

@@ -179,8 +179,12 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* args, void* cuda_st
 /* Same call for callers whose per-step data live in HOST memory: `args` holds HOST pointers
  * for H, draft_tokens, draft_logits and for every output (pinned memory recommended; W stays
  * on the device via jd_set_head). Inputs are copied to handle-owned device staging buffers,
- * the verification runs, the outputs are copied back, and the stream is synchronised before
- * returning. logits_debug must be NULL. */
+ * the verification runs, the outputs are copied back (one copy through a pinned mirror), and the
+ * stream is synchronised before returning. The draft logits, most of the bytes, travel on a second
+ * stream of the handle while the verification already runs; each variant waits for them where it
+ * first reads them (the fused kernel on a device word that the copy's stream sets, with a bounded
+ * wait). Pinned host buffers are needed for that overlap; pageable ones work, serially.
+ * logits_debug must be NULL. */
 jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* args, void* cuda_stream);
 
 /* Synchronises the stream of the handle's last jd_verify and copies the device status word:

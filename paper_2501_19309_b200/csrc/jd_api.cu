@@ -36,6 +36,11 @@ struct jd_handle_s {
   void* st_out;            // accept_len | next_token | judge_scores | p_draft | q_draft | row_max | row_lse | masks
   size_t st_out_bytes;
   void* st_out_host;       // pinned mirror of st_out: the results come back in one copy
+  // host-buffer calls copy the draft logits on the side stream while the verification starts
+  unsigned* dl_flag;       // device word the side stream sets to dl_epoch when the copy has landed
+  unsigned dl_epoch;
+  cudaEvent_t dl_event;    // recorded on the side stream after that copy
+  bool dl_in_flight;       // true only inside jd_verify_host, between enqueueing the copy and jd_verify
 };
 
 namespace {
@@ -72,6 +77,22 @@ bool make_tensor_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t 
   return fn(tm, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+typedef CUresult (*WriteValue32Fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+
+WriteValue32Fn write_value32_fn() {
+  static WriteValue32Fn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (WriteValue32Fn)p;
+  }
+  return fn;
 }
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -124,6 +145,7 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
   w.part_idx = (int*)take(maxR * np * 4);
   w.status = (unsigned*)take(256);
   w.barrier = (unsigned*)take(256);
+  take(256);   // word 0: arrival flag of a host-buffer call's draft logits; outside the per-call memset
   w.np_cap = (int)np;
   w.nq_cap = (int)nq;
   if (ws) *ws = w;
@@ -212,6 +234,11 @@ jd_status_t jd_create(jd_handle_t* out, const jd_config_t* cfg) {
     if (h->side.join) cudaEventDestroy(h->side.join);
     h->side = SideStream{};
   }
+  h->dl_flag = h->ws.barrier + 64;
+  if (h->side.stream && cudaEventCreateWithFlags(&h->dl_event, cudaEventDisableTiming) != cudaSuccess) {
+    cudaGetLastError();
+    h->dl_event = nullptr;
+  }
   *out = h;
   return JD_OK;
 }
@@ -223,6 +250,7 @@ jd_status_t jd_destroy(jd_handle_t h) {
   if (h->side.stream) cudaStreamDestroy(h->side.stream);
   if (h->side.fork) cudaEventDestroy(h->side.fork);
   if (h->side.join) cudaEventDestroy(h->side.join);
+  if (h->dl_event) cudaEventDestroy(h->dl_event);
   cudaFree(h->ws_base);
   cudaFree(h->st_H);
   cudaFree(h->st_x);
@@ -316,6 +344,12 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
     launch_quantize_rows(cp, h->ws, a->H, st);
     launches += 1;
   }
+  if (h->dl_in_flight && variant != JD_VARIANT_FUSED) {
+    // Draft logits still being copied on the side stream: the batched variant reads them there first
+    // (its statistics kernels follow the copy in stream order) and here only after the join; the
+    // CUDA-core variant waits for the copy. The fused kernel is told where to look instead.
+    if (variant == JD_VARIANT_SIMT && cudaStreamWaitEvent(st, h->dl_event, 0) != cudaSuccess) return JD_ERR_CUDA;
+  }
   if (variant == JD_VARIANT_SIMT) {
     launches += run_simt(cp, h->ws, h->W, h->w_scale, h->w_judge, a->H, c.dtype, a->logits_debug, st);
   } else if (variant == JD_VARIANT_BATCHED) {
@@ -341,7 +375,8 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
     if (!make_tensor_map(&tm_h, fp8 ? (const void*)h->ws.h8 : a->H, (uint64_t)R, (uint64_t)c.d, (uint32_t)plan.n_pad, fp8))
       return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
-    const int n = run_fused(cp, h->ws, h->tm_w, tm_h, a->H, h->w_judge, plan, st, &err, false, fp8 ? h->w_scale : nullptr);
+    const int n = run_fused(cp, h->ws, h->tm_w, tm_h, a->H, h->w_judge, plan, st, &err, false, fp8 ? h->w_scale : nullptr,
+                            h->dl_in_flight ? h->dl_flag : nullptr, h->dl_epoch);
     if (n < 0) return JD_ERR_CUDA;
     launches += n;
   }
@@ -389,9 +424,25 @@ jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* a, void* cuda_
   uint8_t* d_mk = (uint8_t*)take(maxBM);
 
   if (cudaMemcpyAsync(h->st_H, a->H, R * c.d * elem_size(c.dtype), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(h->st_x, a->draft_tokens, BM * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(h->st_dl, a->draft_logits, BM * (size_t)c.V * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      cudaMemcpyAsync(h->st_x, a->draft_tokens, BM * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return JD_ERR_CUDA;
+  // The draft logits are most of the bytes. They go over on the side stream, so that the verification
+  // can start as soon as H and the tokens are in; whoever reads them first waits for them (see jd_verify).
+  // Every earlier use of the staging buffer has finished: this function synchronises before it returns.
+  WriteValue32Fn write_value = write_value32_fn();
+  const bool overlap = h->side.stream && h->dl_event && write_value;
+  cudaStream_t dl_stream = overlap ? h->side.stream : st;
+  if (cudaMemcpyAsync(h->st_dl, a->draft_logits, BM * (size_t)c.V * 4, cudaMemcpyHostToDevice, dl_stream) != cudaSuccess)
+    return JD_ERR_CUDA;
+  if (overlap) {
+    h->dl_epoch += 1;
+    if (write_value((CUstream)dl_stream, (CUdeviceptr)(uintptr_t)h->dl_flag, h->dl_epoch, 0) != CUDA_SUCCESS ||
+        cudaEventRecord(h->dl_event, dl_stream) != cudaSuccess) {
+      cudaStreamSynchronize(dl_stream);
+      return JD_ERR_CUDA;
+    }
+    h->dl_in_flight = true;
+  }
 
   jd_verify_args_t dev = *a;
   dev.H = h->st_H; dev.draft_tokens = h->st_x; dev.draft_logits = h->st_dl;
@@ -401,6 +452,10 @@ jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* a, void* cuda_
   dev.row_max = a->row_max ? d_rm : nullptr;
   dev.row_lse = a->row_lse ? d_rl : nullptr;
   jd_status_t s = jd_verify(h, &dev, cuda_stream);
+  if (overlap) {
+    h->dl_in_flight = false;
+    if (s != JD_OK) cudaStreamSynchronize(dl_stream);   // the caller's buffer must not be in use when we return
+  }
   if (s != JD_OK) return s;
 
   // all results in one device-to-host copy (the sections are a few KB), then plain host copies

@@ -52,6 +52,11 @@ struct FusedParams {
   int R;            // rows of the H matrix given to the MMA: B * (M + 1), or B in sample-only mode
   int fp8;          // 1: W and H tiles hold FP8 E4M3 codes (128 per 128-byte row), kind::f8f6f4 MMAs
   int sample_only;  // 1: H holds one already selected row per sequence; only the token draw runs
+  // Host-buffer calls: the draft logits may still be on their way to the device when the kernel
+  // starts. Non-null: the word that the copy's stream sets to dl_epoch once they have arrived;
+  // the epilogue warps wait for it (bounded) before their first read of the draft logits.
+  const unsigned* dl_flag;
+  unsigned dl_epoch;
   uint32_t off_h;   // byte offsets inside dynamic smem (from the 1024-aligned base)
   uint32_t off_ovf;
   uint32_t off_w;
@@ -318,6 +323,25 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
 
     // (b) while W streams: draft-row statistics over this CTA's vocabulary slice, judge dots
+    if (fp.dl_flag != nullptr) {   // draft logits still in flight: wait for the copy stream's signal
+      if (tid == 0) {
+        bool arrived = false;
+        for (unsigned it = 0; it < kSpinLimit / 4 && !arrived; ++it) {
+          unsigned v;
+          asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(fp.dl_flag) : "memory");
+          arrived = (v == fp.dl_epoch);
+          if (!arrived) {
+            if (*abort_flag) break;
+            __nanosleep(100);
+          }
+        }
+        if (!arrived) {
+          *abort_flag = 1;
+          set_status(ws.status, JD_ERR_TIMEOUT);
+        }
+      }
+      epi_sync();
+    }
     const int v_lo = t0 * kVocabTile, v_hi = min(V, (t0 + T) * kVocabTile);
     const bool vec4 = (V % 4) == 0;   // rows are 16-byte aligned only then
     for (int bm = warp; bm < (fp.sample_only ? 0 : BM); bm += 4) {
@@ -330,7 +354,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int v = v_lo + (i0 + u) * kVocabTile + lane * 4;
-            x[u] = (i0 + u < T && v < V) ? __ldg(reinterpret_cast<const float4*>(row + v))
+            x[u] = (i0 + u < T && v < V) ? __ldcg(reinterpret_cast<const float4*>(row + v))
                                          : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
           }
           float mm = -INFINITY;
@@ -350,7 +374,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
       } else {
         for (int v = v_lo + lane; v < v_hi; v += 32) {
-          const float xv = __ldg(row + v);
+          const float xv = __ldcg(row + v);
           if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
           else if (xv != -INFINITY) s += __expf(xv - m);
         }
@@ -361,7 +385,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         ws.qpart_sum[(size_t)bm * G + cta] = s;
         const int b = bm / M, j = bm % M;
         const int x = ms.x_row[b * (M + 1) + j];
-        if (x >= v_lo && x < v_hi) ws.qgath[bm] = row[x];
+        if (x >= v_lo && x < v_hi) ws.qgath[bm] = __ldcg(row + x);
       }
     }
     for (int bm = cta * 4 + warp; bm < (fp.sample_only ? 0 : BM); bm += G * 4) {
@@ -712,7 +736,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
               const int vg = (t0 + i0 + u) * kVocabTile + tid;
-              dv[q][u] = (kind == 0 && b0 + q < cp.B && i0 + u < T && vg < V) ? __ldg(dlrow + vg) : 0.f;
+              dv[q][u] = (kind == 0 && b0 + q < cp.B && i0 + u < T && vg < V) ? __ldcg(dlrow + vg) : 0.f;
             }
           }
 #pragma unroll
@@ -857,7 +881,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
             const float* src = fp.sample_only ? ws.w_sel + ((size_t)(t0 + i0 + u) * cp.B + b) * kVocabTile + tid
                                               : dlrow + vg;
-            dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldg(src) : 0.f;
+            dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldcg(src) : 0.f;
           }
           load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], &ms.swt[0][0], lg);
 #pragma unroll
@@ -1001,8 +1025,10 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
 
 int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
               const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err,
-              bool sample_only, const float* w_scale_fp8) {
+              bool sample_only, const float* w_scale_fp8, const unsigned* dl_flag, unsigned dl_epoch) {
   FusedParams fp;
+  fp.dl_flag = sample_only ? nullptr : dl_flag;
+  fp.dl_epoch = dl_epoch;
   fp.fp8 = w_scale_fp8 ? 1 : 0;
   fp.num_kb = cp.d / (fp.fp8 ? kBlockK8 : kBlockK);
   fp.num_tiles = (cp.V + kVocabTile - 1) / kVocabTile;

@@ -542,3 +542,38 @@ def test_two_handles_on_two_streams_do_not_disturb_each_other():
         for k in want:
             assert np.array_equal(want[k], got[k]), k
         ver.close()
+
+
+@pytest.mark.parametrize("variant,B,M,d,V,dtype,pinned", [
+    ("simt", 3, 5, 100, 4000, "bf16", True),       # the copy of the draft logits is waited for by an event
+    ("fused", 2, 12, 128, 128256, "bf16", True),   # ... by the kernel itself, on a flag the copy's stream sets
+    ("fused", 2, 12, 128, 128256, "bf16", False),  # pageable buffers: the copy is staged, nothing overlaps
+    ("batched", 20, 6, 128, 60000, "bf16", True),  # ... by stream order on the side stream
+    ("batched", 100, 2, 128, 9000, "fp8", True),
+])
+def test_host_call_with_draft_logits_in_flight(variant, B, M, d, V, dtype, pinned):
+    """jd_verify_host copies the draft logits on a second stream while the verification starts; every
+    variant must wait for them where it first reads them, call after call, with changing inputs."""
+    import torch
+    wl = I.CONFIGS[2].scaled("inflight-" + variant, B=B, M=M, d=d, V=V, dtype=dtype)
+    ver = None
+    for data_seed in (50, 51, 52):
+        inp = I.make_inputs(wl, data_seed)
+        dev = T.upload(inp)
+        if ver is None:
+            ver = T.make_verifier(inp, dev)
+        else:
+            ver.set_head(dev["W"], dev["w"], inp.b_judge, w_scale=dev.get("w_scale"))
+        want = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, data_seed, "judge_or_standard", variant=variant))
+        hH = torch.from_numpy(inp.H).view(torch.bfloat16)
+        hx = torch.from_numpy(inp.draft_tokens)
+        hdl = torch.from_numpy(inp.draft_logits)
+        if pinned:
+            hH, hx, hdl = hH.pin_memory(), hx.pin_memory(), hdl.pin_memory()
+        got = ver.verify_host(hH, hx, hdl, 0.5, data_seed, "judge_or_standard", variant=variant)
+        got = {k: v.numpy().copy() for k, v in got.items()}
+        from paper_2501_19309_b200 import jd
+        assert ver.device_status() == jd.JD_OK
+        for k in want:
+            assert np.array_equal(want[k], got[k]), (variant, data_seed, k)
+    ver.close()

@@ -33,7 +33,6 @@ namespace jd {
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int kEpiThreads = 128;
 constexpr int kBlockK = 64;                      // bf16 elements per k-slice = one 128-byte swizzle row
 constexpr int kBlockK8 = 128;                    // FP8 codes per k-slice (same 128 bytes)
 constexpr int kWStageBytes = kVocabTile * 128;   // 16 KB

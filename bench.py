@@ -58,7 +58,7 @@ class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, gpu_index: int):
         self.proc = None
@@ -79,7 +79,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
             out = ""
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.strip().splitlines():
             f = [t.strip() for t in line.split(",")]
@@ -93,8 +93,12 @@ class ClockSampler:
             for n, v in zip(names, f[2:6]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
+            try:
+                pw.append(float(f[6]))
+            except (IndexError, ValueError):
+                pass
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "power_w": statistics.median(pw) if pw else None}
 
 
 def max_over_ranks(values, device, dist_on: bool):
@@ -121,6 +125,9 @@ def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, 
         bytes_alg = wl.V * wl.d + wl.V * 4 + wl.R * wl.d * 2
     else:
         bytes_alg = wl.V * wl.d * 2 + wl.R * wl.d * 2        # W once + H once
+    # everything the call must move: + the draft logits once for their statistics and one row per sequence
+    # again for the residual, tokens in, results out (the metric's own byte count leaves these out)
+    bytes_all = bytes_alg + wl.B * wl.M * wl.V * 4 + wl.B * wl.V * 4 + wl.B * wl.M * 4 + wl.B * (8 + 8 * wl.M)
     flops = 2.0 * wl.R * wl.V * wl.d
     tf_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
     tf_sustained = peaks["bf16_tflops_sustained"]
@@ -135,12 +142,14 @@ def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, 
                 "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "peak_source": which,
                 "frac_of_nominal_peak": ach / NOMINAL_HBM_GBS,
                 "read_stream_gbs": stream_gbs, "frac_of_read_stream": ach / stream_gbs if stream_gbs else None,
-                "algorithmic_bytes": bytes_alg, "kernel_ms": kernel_ms}
+                "algorithmic_bytes": bytes_alg, "all_bytes": bytes_all,
+                "frac_all_bytes": bytes_all / (kernel_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "kernel_ms": kernel_ms}
     ach = flops / (kernel_ms * 1e-3) / 1e12
     return {"bound": "tensor", "achieved": ach, "peak": tf_peak, "unit": "TFLOP/s", "frac": ach / tf_peak,
             "frac_of_sustained_peak": ach / tf_sustained,
             "frac_of_nominal_peak": ach / (NOMINAL_BF16_TFLOPS * (2 if wl.dtype == "fp8" else 1)),
-            "traffic": traffic, "peak_source": which, "algorithmic_flops": flops, "kernel_ms": kernel_ms}
+            "traffic": traffic, "peak_source": which, "algorithmic_flops": flops, "all_bytes": bytes_all,
+            "kernel_ms": kernel_ms}
 
 
 def oracle_step(inp: I.Inputs, seed: int, sequences):
@@ -382,12 +391,13 @@ def main() -> None:
                 owl = owl.scaled(owl.name + "-fp8", dtype="fp8")
             small.steps = max(50, min(args.steps, 300))
             small.e2e_steps = 10
-            r = measure_workload(owl, small, torch, jd, device, data_seed=0, sample_clocks=False)
+            r = measure_workload(owl, small, torch, jd, device, data_seed=0, sample_clocks=True)
             others[owl.name] = {
                 "B": owl.B, "M": owl.M, "d": owl.d, "V": owl.V, "ms_per_step": r["mean_ms"],
                 "median_ms": r["median_ms"], "value": owl.B * owl.M / (r["mean_ms"] * 1e-3), "unit": UNIT,
                 "variant": VARIANT_NAMES.get(r["variant"], "?"), "kernel_launches_per_step": r["launches"],
                 "steps": small.steps, "mean_accept_len": r["mean_accept"], "best_ms": r["min_ms"],
+                "clocks": r["clocks"],
                 "graph_replay_ms_per_step": r["graph_ms"],
                 "emitted_tokens_per_s": r["emitted_per_call"] / (r["mean_ms"] * 1e-3),
                 "e2e_value": owl.B * owl.M * r["e2e_steps"] / r["e2e_s"],

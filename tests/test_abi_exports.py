@@ -44,3 +44,19 @@ def test_struct_layout_matches_header_order():
     body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
     fields = re.findall(r"([A-Za-z_0-9]+)\s*;", body)
     assert fields == [f[0] for f in jd.jd_verify_args_t._fields_]
+
+
+def test_header_and_c_caller_compile_as_plain_c():
+    """include/jd.h is a C header: the C99 caller under tests/c_abi builds with gcc, warnings as errors."""
+    import shutil
+    import subprocess
+    import tempfile
+    cuda_inc = "/usr/local/cuda/include"
+    if shutil.which("gcc") is None or not os.path.exists(os.path.join(cuda_inc, "cuda_runtime_api.h")):
+        import pytest
+        pytest.skip("gcc or the CUDA runtime header is not installed")
+    with tempfile.TemporaryDirectory() as tmp:
+        cmd = ["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(ROOT, "include"), "-I", cuda_inc,
+               "-c", os.path.join(ROOT, "tests", "c_abi", "jd_c_caller.c"), "-o", os.path.join(tmp, "caller.o")]
+        proc = subprocess.run(cmd, capture_output=True, text=True)
+        assert proc.returncode == 0, proc.stderr

@@ -577,3 +577,55 @@ def test_host_call_with_draft_logits_in_flight(variant, B, M, d, V, dtype, pinne
         for k in want:
             assert np.array_equal(want[k], got[k]), (variant, data_seed, k)
     ver.close()
+
+
+# ------------------------------------------------------------------ the C ABI from C
+def test_plain_c_program_calls_the_library():
+    """tests/c_abi/jd_c_caller.c (C99, gcc, no Python or torch in the process) runs one host-buffer
+    verification through the C ABI; its outputs are checked against the CPU checker like any other."""
+    import os
+    import shutil
+    import struct
+    import subprocess
+    import tempfile
+    from paper_2501_19309_b200 import jd
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    cuda = "/usr/local/cuda"
+    if shutil.which("gcc") is None or not os.path.exists(cuda + "/lib64/libcudart.so"):
+        pytest.skip("gcc or libcudart is not installed")
+    wl = I.CONFIGS[2].scaled("c-caller", B=3, M=7, d=128, V=40000)
+    inp = I.make_inputs(wl, 61)
+    mode = "judge_or_standard"
+    libdir = os.path.dirname(jd.library_path())
+    with tempfile.TemporaryDirectory() as tmp:
+        exe, prob, res = (os.path.join(tmp, n) for n in ("caller", "problem.bin", "result.bin"))
+        build = ["gcc", "-std=c99", "-O1", "-I", os.path.join(root, "include"), "-I", cuda + "/include",
+                 os.path.join(root, "tests", "c_abi", "jd_c_caller.c"), "-o", exe, "-L", libdir, "-ljd_b200",
+                 "-L", cuda + "/lib64", "-lcudart", "-Wl,-rpath," + libdir, "-Wl,-rpath," + cuda + "/lib64"]
+        proc = subprocess.run(build, capture_output=True, text=True)
+        assert proc.returncode == 0, proc.stderr
+        with open(prob, "wb") as f:
+            f.write(struct.pack("<5i2fQ", wl.B, wl.M, wl.d, wl.V, jd.MODES[mode], inp.tau, inp.b_judge, inp.seed))
+            for a in (inp.W, inp.w_judge, inp.H, inp.draft_tokens, inp.draft_logits):
+                f.write(np.ascontiguousarray(a).tobytes())
+        proc = subprocess.run([exe, prob, res], capture_output=True, text=True, timeout=300)
+        assert proc.returncode == 0, proc.stderr
+        raw = open(res, "rb").read()
+    B, M, R = wl.B, wl.M, wl.B * (wl.M + 1)
+    off = 0
+
+    def take(dtype, n):
+        nonlocal off
+        a = np.frombuffer(raw, dtype=dtype, count=n, offset=off)
+        off += a.nbytes
+        return a
+    status, variant, launches = take(np.int32, 3)
+    assert status == jd.JD_OK and variant == jd.JD_VARIANT_FUSED and launches >= 1
+    got = dict(accept_len=take(np.int32, B), next_token=take(np.int32, B),
+               judge_scores=take(np.float32, B * M).reshape(B, M), p_draft=take(np.float32, B * M).reshape(B, M),
+               q_draft=take(np.float32, B * M).reshape(B, M), masks=take(np.uint8, B * M).reshape(B, M),
+               row_max=take(np.float32, R).reshape(B, M + 1), row_lse=take(np.float32, R).reshape(B, M + 1))
+    assert off == len(raw)
+    ref = T.run_oracle(inp, mode)
+    rep = T.compare(got, ref, mode, M)
+    assert rep.sequences == B

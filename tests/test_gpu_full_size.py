@@ -108,3 +108,17 @@ def test_cfg3_fp8_head_full_size():
 def test_cfg4_fp8_head_sampled_sequences():
     rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[0, 63], expect_variant="batched", fp8=True)
     assert rep.sequences == 2
+
+
+@pytest.mark.parametrize("data_seed", [2, 3, 4, 5, 6, 7, 8, 9])
+def test_cfg1_remaining_seeds(data_seed):
+    """Seeds 0 and 1 run the whole threshold sweep above; the other eight of the workload's ten seeds
+    (data seed = verify seed) run the paper's mode at tau = 0.5."""
+    full_case(1, data_seed, [("judge_or_standard", 0.5)], expect_variant="fused")
+
+
+@pytest.mark.parametrize("data_seed", [1, 2, 3, 4])
+def test_cfg4_remaining_seeds_one_sequence_each(data_seed):
+    rep, _ = full_case(4, data_seed, [("judge_or_standard", None)], sequences=[(17 * data_seed) % 64],
+                       expect_variant="batched")
+    assert rep.sequences == 1

@@ -31,6 +31,7 @@ struct FusedPlan {
   int tile_stride;    // TMEM columns between consecutive tiles
   size_t smem_bytes;  // dynamic shared memory of the launch
   int stages;         // W ring depth
+  int h_stages;       // H ring depth
 };
 void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st);
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan);

@@ -17,8 +17,9 @@
 // exactly once and H is re-read (from L2) once per group, not once per tile.
 // Where the statistics passes are long enough to matter (see run_fused), a CTA whose tiles all
 // fit in TMEM sweeps d twice: first over all tiles but the last, then over the last one. The
-// epilogue warps take the row statistics of the early tiles while the last tile still streams,
-// so only one tile's worth of statistics is left for the time after the stream.
+// epilogue warps take the row statistics of the early tiles (in sample-only mode: their sampling
+// masses) while the last tile still streams, so only one tile's worth is left for the time after
+// the stream.
 //
 // After the main loop the grid meets twice:
 //   per-CTA (max, sum exp) of every row, logit of the drafted tokens        -> barrier 1
@@ -234,7 +235,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   // TMEM-resident tiles, which reuse the columns the overflow tiles have left. Without overflow
   // and with late_tiles set: group 0 = the first T_early tiles, group 1 = the rest, every tile in
   // columns of its own; the statistics of group 0 are taken while group 1 streams.
-  const int T_early = (n_ovf == 0 && !fp.sample_only && fp.late_tiles > 0 && T > fp.late_tiles + 1) ? T - fp.late_tiles : 0;
+  const int T_early = (n_ovf == 0 && fp.late_tiles > 0 && T > fp.late_tiles + 1) ? T - fp.late_tiles : 0;
   const int g_split = n_ovf > 0 ? n_ovf : T_early;
   const int g_begin[2] = {0, g_split};
   const int g_end[2] = {g_split, T};
@@ -426,13 +427,89 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     // starts when the whole accumulation is complete. A CTA that ran an early sweep (T_early > 0)
     // first takes, in phase 0, the statistics of the early tiles while the last sweep still streams,
     // and merges the two (max, sum exp) pairs per row at the end.
+    if (fp.sample_only) {
+      // an earlier kernel made the decisions; fetch what the token draw needs
+      if (tid < cp.B) {
+        ms.sel_row[tid] = ws.sel_row[tid];
+        ms.sel_kind[tid] = ws.sel_kind[tid];
+        ms.sel_lse_p[tid] = ws.sel_lse_p[tid];
+        ms.sel_lse_q[tid] = ws.sel_lse_q[tid];
+        ms.sel_u[tid] = ws.sel_u[tid];
+      }
+      epi_sync();
+    }
     for (int ph = (T_early > 0 ? 0 : 1); ph < 2; ++ph) {
       if (tid == 0 && ok && (ph == 0 || T > n_ovf)) mbar_wait(smem_u32(&ms.acc_full[ph]), 0u, abort_flag);
       epi_sync();
       tc_fence_after();
       ok = ok && (*abort_flag == 0);
-      if (fp.sample_only) continue;
       const int i_lo = ph == 0 ? 0 : T_early, i_hi = ph == 0 ? T_early : T;
+      if (fp.sample_only) {
+        // (h) mass of the sampling weights of each selected row over the phase's tiles.
+        // Sample-only mode: every TMEM column is a selected row, so the tiles are read 16 columns
+        // (= 16 sequences) at a time, like the statistics passes.
+        if (ok && cp.rule != JD_RULE_TOPK) {
+#pragma unroll
+          for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+            if (c0 >= cp.B) break;
+            // A thread adds at most a handful of tiles per sequence, so its own partial sums stay in
+            // fp32 (32 double accumulators would not fit in registers); everything summed across
+            // lanes, warps and CTAs is double. The loop body is branch-free: with one warp per
+            // scheduler, branches around each sequence would serialise sixteen latency chains.
+            float sr[16], sp[16], lp2[16], lq2[16];
+            int kd[16];   // 0: residual, 1: p alone, 2: column past the last sequence
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+              const int b = min(c0 + k, cp.B - 1);
+              sr[k] = 0.f; sp[k] = 0.f;
+              kd[k] = (c0 + k < cp.B) ? ms.sel_kind[b] : 2;
+              lp2[k] = ms.sel_lse_p[b] * kLog2e;
+              lq2[k] = ms.sel_lse_q[b] * kLog2e;
+            }
+            const int last_tile = fp.num_tiles - 1;
+            for (int i0 = i_lo; i0 < i_hi; i0 += 2) {
+              const int vg0 = (t0 + i0) * kVocabTile + tid, vg1 = vg0 + kVocabTile;
+              const bool val0 = vg0 < V, val1 = (i0 + 1 < i_hi) && vg1 < V;
+              // ws.w_sel holds the selected draft rows tile-major, [vocab tile][sequence][128]: this
+              // CTA's share is one contiguous block. Rows that need no residual were not gathered;
+              // what is read for them is discarded by the select below.
+              const float* base0 = ws.w_sel + ((size_t)(t0 + i0) * cp.B + min(c0, cp.B - 1)) * kVocabTile + tid;
+              const float* base1 = ws.w_sel + ((size_t)min(t0 + i0 + 1, last_tile) * cp.B + min(c0, cp.B - 1)) * kVocabTile + tid;
+              float d0[16], d1[16], v0[16], v1[16];
+#pragma unroll
+              for (int k = 0; k < 16; ++k) {
+                const int kk = min(k, cp.B - 1 - min(c0, cp.B - 1));   // stay inside the buffer in a ragged last chunk
+                d0[k] = __ldg(base0 + kk * kVocabTile);
+                d1[k] = __ldg(base1 + kk * kVocabTile);
+              }
+              load_chunk2<N_PAD>(i0, i_hi, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0], v0, v1);
+#pragma unroll
+              for (int k = 0; k < 16; ++k) {
+                const float p0 = fast_exp2(fmaf(v0[k], kLog2e, -lp2[k])), q0 = fast_exp2(fmaf(d0[k], kLog2e, -lq2[k]));
+                const float p1 = fast_exp2(fmaf(v1[k], kLog2e, -lp2[k])), q1 = fast_exp2(fmaf(d1[k], kLog2e, -lq2[k]));
+                const float r0 = kd[k] == 0 ? fmaxf(0.f, p0 - q0) : p0;
+                const float r1 = kd[k] == 0 ? fmaxf(0.f, p1 - q1) : p1;
+                const bool on0 = val0 && kd[k] < 2, on1 = val1 && kd[k] < 2;
+                sr[k] += (on0 ? r0 : 0.f) + (on1 ? r1 : 0.f);
+                sp[k] += (on0 ? p0 : 0.f) + (on1 ? p1 : 0.f);
+              }
+            }
+            double dsum[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) dsum[k] = (double)sr[k];
+            const double red_r = warp_reduce16<false, double>(dsum, lane);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) dsum[k] = (double)sp[k];
+            const double red_p = warp_reduce16<false, double>(dsum, lane);
+            const int bq = c0 + reduce16_index(lane);
+            if ((lane & 1) == 0 && bq < cp.B) {
+              if (ph == 1 && T_early > 0) { ms.wd_r[bq][warp] += red_r; ms.wd_p[bq][warp] += red_p; }   // same thread wrote phase 0
+              else { ms.wd_r[bq][warp] = red_r; ms.wd_p[bq][warp] = red_p; }
+            }
+          }
+        }
+        continue;
+      }
 
       // (d) gather of the drafted tokens' logits (rows listed in the prologue), per-row max
       if (ok && ph == 1) {
@@ -660,16 +737,6 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     epi_sync();
 
-    } else {
-      // sample-only mode: an earlier kernel made the decisions; fetch what the token draw needs
-      if (ok && tid < cp.B) {
-        ms.sel_row[tid] = ws.sel_row[tid];
-        ms.sel_kind[tid] = ws.sel_kind[tid];
-        ms.sel_lse_p[tid] = ws.sel_lse_p[tid];
-        ms.sel_lse_q[tid] = ws.sel_lse_q[tid];
-        ms.sel_u[tid] = ws.sel_u[tid];
-      }
-      epi_sync();
     }
 
     // top-K rule: the next token is the argmax of the selected row; CTA 0 folds the per-CTA maxima
@@ -699,66 +766,8 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
     }
 
-    // (h) mass of the sampling weights of each selected row over this CTA's slice.
-    // Sample-only mode: every TMEM column is a selected row, so the tiles are read 16 columns
-    // (= 16 sequences) at a time, like the statistics passes.
-    if (ok && draw && fp.sample_only) {
-#pragma unroll
-      for (int c0 = 0; c0 < N_PAD; c0 += 16) {
-        if (c0 >= cp.B) break;
-        // A thread adds at most a handful of tiles per sequence, so its own partial sums stay in
-        // fp32 (32 double accumulators would not fit in registers); everything summed across
-        // lanes, warps and CTAs is double. The loop body is branch-free: with one warp per
-        // scheduler, branches around each sequence would serialise sixteen latency chains.
-        float sr[16], sp[16], lp2[16], lq2[16];
-        int kd[16];   // 0: residual, 1: p alone, 2: column past the last sequence
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const int b = min(c0 + k, cp.B - 1);
-          sr[k] = 0.f; sp[k] = 0.f;
-          kd[k] = (c0 + k < cp.B) ? ms.sel_kind[b] : 2;
-          lp2[k] = ms.sel_lse_p[b] * kLog2e;
-          lq2[k] = ms.sel_lse_q[b] * kLog2e;
-        }
-        const int last_tile = fp.num_tiles - 1;
-        for (int i0 = 0; i0 < T; i0 += 2) {
-          const int vg0 = (t0 + i0) * kVocabTile + tid, vg1 = vg0 + kVocabTile;
-          const bool val0 = vg0 < V, val1 = (i0 + 1 < T) && vg1 < V;
-          // ws.w_sel holds the selected draft rows tile-major, [vocab tile][sequence][128]: this
-          // CTA's share is one contiguous block. Rows that need no residual were not gathered;
-          // what is read for them is discarded by the select below.
-          const float* base0 = ws.w_sel + ((size_t)(t0 + i0) * cp.B + min(c0, cp.B - 1)) * kVocabTile + tid;
-          const float* base1 = ws.w_sel + ((size_t)min(t0 + i0 + 1, last_tile) * cp.B + min(c0, cp.B - 1)) * kVocabTile + tid;
-          float d0[16], d1[16], v0[16], v1[16];
-#pragma unroll
-          for (int k = 0; k < 16; ++k) {
-            const int kk = min(k, cp.B - 1 - min(c0, cp.B - 1));   // stay inside the buffer in a ragged last chunk
-            d0[k] = __ldg(base0 + kk * kVocabTile);
-            d1[k] = __ldg(base1 + kk * kVocabTile);
-          }
-          load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0], v0, v1);
-#pragma unroll
-          for (int k = 0; k < 16; ++k) {
-            const float p0 = fast_exp2(fmaf(v0[k], kLog2e, -lp2[k])), q0 = fast_exp2(fmaf(d0[k], kLog2e, -lq2[k]));
-            const float p1 = fast_exp2(fmaf(v1[k], kLog2e, -lp2[k])), q1 = fast_exp2(fmaf(d1[k], kLog2e, -lq2[k]));
-            const float r0 = kd[k] == 0 ? fmaxf(0.f, p0 - q0) : p0;
-            const float r1 = kd[k] == 0 ? fmaxf(0.f, p1 - q1) : p1;
-            const bool on0 = val0 && kd[k] < 2, on1 = val1 && kd[k] < 2;
-            sr[k] += (on0 ? r0 : 0.f) + (on1 ? r1 : 0.f);
-            sp[k] += (on0 ? p0 : 0.f) + (on1 ? p1 : 0.f);
-          }
-        }
-        double dsum[16];
-#pragma unroll
-        for (int k = 0; k < 16; ++k) dsum[k] = (double)sr[k];
-        const double red_r = warp_reduce16<false, double>(dsum, lane);
-#pragma unroll
-        for (int k = 0; k < 16; ++k) dsum[k] = (double)sp[k];
-        const double red_p = warp_reduce16<false, double>(dsum, lane);
-        const int bq = c0 + reduce16_index(lane);
-        if ((lane & 1) == 0 && bq < cp.B) { ms.wd_r[bq][warp] = red_r; ms.wd_p[bq][warp] = red_p; }
-      }
-    }
+    // (h) mass of the sampling weights of each selected row over this CTA's slice (sample-only mode:
+    // done above, phase by phase, as the tiles completed).
     // Full mode: the few selected rows sit in scattered columns; four sequences at a time so
     // that their draft-logit loads are in flight together.
     if (ok && draw && !fp.sample_only) {
@@ -1087,7 +1096,10 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
   // Early sweep + one late tile: measured on B200 over 16 to 80 padded rows and d = 4096 to 16384,
   // it shortens the call by 2-4 % once the statistics passes are long enough to be worth hiding
   // (48 padded rows or more, or 32 with at least 128 k-steps) and lengthens it by 1-5 % below that.
-  fp.late_tiles = (!sample_only && (plan.n_pad >= 48 || (plan.n_pad >= 32 && fp.num_kb >= 128))) ? 1 : 0;
+  // In sample-only mode the early tiles' sampling masses are what the last sweep hides: 1-5 % shorter
+  // batched calls at 16 to 64 sequences.
+  fp.late_tiles = sample_only ? 1
+                              : ((plan.n_pad >= 48 || (plan.n_pad >= 32 && fp.num_kb >= 128)) ? 1 : 0);
   fp.off_h = kMiscBytes;
   fp.off_ovf = fp.off_h + plan.h_stages * plan.n_pad * 128;
   const int n_ovf = plan.max_tiles - plan.tmem_tiles;

@@ -185,7 +185,10 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const int R = fp.R, M = cp.M, V = cp.V;
   const int BM = cp.B * M;
 
-  if (tid == 0) {
+  // The producer warp sets up the barriers and leaves the prologue without waiting for the other
+  // warps (it arrives at the block's hand-over barrier, they wait on it), so that W starts to
+  // stream while they still fetch the drafted tokens and allocate tensor memory.
+  if (warp == 4 && lane == 0) {
     for (int s = 0; s < fp.stages; ++s) { mbar_init(smem_u32(&ms.full_w[s]), 1); mbar_init(smem_u32(&ms.empty_w[s]), 1); }
     for (int s = 0; s < fp.h_stages; ++s) { mbar_init(smem_u32(&ms.full_h[s]), 1); mbar_init(smem_u32(&ms.empty_h[s]), 1); }
     mbar_init(smem_u32(&ms.acc_full[0]), 1);
@@ -223,9 +226,14 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
-  __syncthreads();
+  if (warp == 4) {
+    __syncwarp();
+    asm volatile("bar.arrive 2, 192;" ::: "memory");
+  } else {
+    asm volatile("bar.sync 2, 192;" ::: "memory");
+  }
   tc_fence_after();
-  const uint32_t tmem_base = ms.tmem_base;
+  const uint32_t tmem_base = ms.tmem_base;   // (not meaningful in the producer warp, which does not use it)
   if (tid < R) {   // rows whose drafted token this CTA's slice holds (usually none or one)
     const int x = ms.x_row[tid];
     if (x >= t0 * kVocabTile && x < (t0 + T) * kVocabTile) ms.glist[atomicAdd(&ms.glist_n, 1)] = tid;

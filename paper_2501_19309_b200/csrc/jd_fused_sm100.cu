@@ -5,8 +5,8 @@
 // (TMEM columns) the rows of H. D[v, r] = sum_k W[v, k] H[r, k]. Each CTA owns a contiguous
 // range of 128-entry vocabulary tiles (at most seven for V = 128256 on 148 SMs) and keeps the
 // fp32 logits of ALL of them on chip until the call ends: tile i occupies TMEM columns
-// [i*N_PAD, (i+1)*N_PAD); tiles that do not fit in the 512 columns are computed first and moved
-// to shared memory. The logits never reach device memory.
+// [i*S, i*S + rows), S = rows rounded up to 8; tiles that do not fit in the 512 columns are
+// computed first and moved to shared memory. The logits never reach device memory.
 //
 // Warp roles (192 threads): warps 0-3 statistics / decisions / sampling (one TMEM lane
 // quadrant each), warp 4 lane 0 TMA producer, warp 5 lane 0 MMA issuer (warp 5 owns the TMEM
@@ -21,12 +21,13 @@
 // masses) while the last tile still streams, so only one tile's worth is left for the time after
 // the stream.
 //
-// After the main loop the grid meets twice:
-//   per-CTA (max, sum exp) of every row, logit of the drafted tokens        -> barrier 1
-//   every CTA folds the statistics, runs the tests and the prefix rule (identical results),
-//   then computes its slice of the sampling mass of each sequence's selected row -> barrier 2
+// After the main loop the grid meets three times:
+//   per-CTA (max, sum exp) of every row, logit of the drafted tokens            -> barrier 1
+//   the rows' partials are folded, each CTA taking a share of the rows          -> barrier 2
+//   every CTA runs the tests and the prefix rule (identical results), then computes its slice
+//   of the sampling mass of each sequence's selected row                        -> barrier 3
 //   the CTA whose slice contains T = u * total mass locates the token.
-// Both barriers are counters in global memory, legal because the launch is cooperative (all
+// The barriers are counters in global memory, legal because the launch is cooperative (all
 // CTAs co-resident); every wait in the kernel is bounded and reports JD_ERR_TIMEOUT.
 #include <cooperative_groups.h>
 

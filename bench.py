@@ -38,8 +38,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes (read + write) per verification call from the ncu captures summarised under profiles/
 # (dominant kernels of each workload); set an entry to None when its kernel changes.
-NCU_TRAFFIC_BYTES = {"cfg1-8B-head": None, "cfg2-70B-head": None, "cfg3-405B-head": None,
-                     "cfg3-405B-head-fp8": None, "cfg4-batched": None, "cfg4-batched-fp8": None}
+NCU_TRAFFIC_BYTES = {"cfg1-8B-head": 1.0593e9, "cfg2-70B-head": 2.1576e9, "cfg3-405B-head": 4.2244e9,
+                     "cfg3-405B-head-fp8": 2.1230e9,
+                     "cfg4-batched": 2.1495e9 + 2.1448e9,          # GEMM pass + second pass
+                     "cfg4-batched-fp8": 1.0666e9 + 1.0905e9}
 VARIANT_NAMES = {1: "simt", 2: "fused", 3: "batched"}
 
 

@@ -38,10 +38,10 @@ normalisation gain is taken as folded into W beforehand.
 
 8-bit head (the paper runs its targets with 8-bit weights, Table 1 caption and App. B.3): with
 w_scale given, W holds FP8 E4M3 codes (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no
-infinities) and the logical weight is w_scale[v] * e4m3(W[v,k]). The rows of H are then quantised
-the same way before the LM head: s_r = max_k |H[r,k]| / 448 and h8 = e4m3(round-to-nearest-even,
-saturating, of H[r,k] * (448 / max_k |H[r,k]|)), the scale and the product in float32 as the
-kernel takes them, so that both sides pick the same codes. The logit is
+infinities) and the logical weight is w_scale[v] * e4m3(W[v,k]). The rows of H are quantised the
+same way before the LM head, one scale per row: with a_r = max_k |H[r,k]|, the scale is
+s_r = a_r / 448 and h8[r,k] is the E4M3 value nearest to H[r,k] * 448 / a_r (ties to the even
+mantissa, saturating at +-448; an all-zero row gives zeros and s_r = 0). The logit is
 w_scale[v] * s_r * sum_k e4m3(W[v,k]) * h8[r,k]; the judge still reads the unquantised row.
 
 Readings taken where the paper is silent (all restated in the design notes):
@@ -151,27 +151,26 @@ def e4m3_decode(codes: np.ndarray) -> np.ndarray:
 
 
 def e4m3_round(x: np.ndarray) -> np.ndarray:
-    """Nearest E4M3 value of every float32 in x, ties to even, saturating at +-448; float64."""
-    x = np.asarray(x, dtype=np.float32).astype(np.float64)
+    """Nearest E4M3 value of every entry of x (float64), ties to the even mantissa, saturating at
+    +-448; float64."""
+    x = np.asarray(x, dtype=np.float64)
     a = np.minimum(np.abs(x), 448.0)
     # spacing of the E4M3 grid around a: 2^(floor(log2 a) - 3), but never finer than 2^-9
     ex = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))
     q = np.ldexp(1.0, (ex - 3).astype(np.int64))
-    r = np.round(a / q) * q                   # numpy rounds halves to even; a / q is exact
+    r = np.round(a / q) * q                   # numpy rounds halves to even; a / q is exact (q = 2^n)
     return np.copysign(np.minimum(r, 448.0), x)
 
 
 def quantise_rows_e4m3(Hb: np.ndarray) -> tuple:
-    """Per-row E4M3 quantisation in the kernel's arithmetic: returns (values [rows, d] float64 on
-    the E4M3 grid, scale [rows] float64) with H ~ scale * values."""
-    Hf = _to_f64(Hb).astype(np.float32)                    # bf16 / f32 inputs are exact in float32
-    amax = np.max(np.abs(Hf), axis=-1, keepdims=True).astype(np.float32)
-    safe = np.where(amax > 0, amax, np.float32(1.0)).astype(np.float32)
-    inv = (np.float32(448.0) / safe).astype(np.float32)    # float32 division, round to nearest
-    scaled = (Hf * inv).astype(np.float32)                 # float32 product, round to nearest
-    vals = e4m3_round(scaled)
-    scale = (amax / np.float32(448.0)).astype(np.float32)  # float32 division
-    return vals, scale[..., 0].astype(np.float64)
+    """Per-row E4M3 quantisation: returns (values [rows, d] float64 on the E4M3 grid, scale [rows]
+    float64) with H ~ scale * values; scale = row amax / 448, values = nearest E4M3 value of
+    H * 448 / amax."""
+    Hd = _to_f64(Hb)
+    amax = np.max(np.abs(Hd), axis=-1, keepdims=True)
+    safe = np.where(amax > 0, amax, 1.0)
+    vals = e4m3_round(Hd * 448.0 / safe)       # H * 448 is exact in float64 for bf16 / f32 inputs
+    return vals, (amax / 448.0)[..., 0]
 
 
 def rms_normalise(Hb: np.ndarray, eps: float) -> np.ndarray:

@@ -9,6 +9,14 @@ synthetic draft block.  Prints ONE JSON line:
   roofline  achieved (W bytes + H bytes) / kernel time against the measured HBM copy bandwidth
             (or 2*R*V*d flop / time against the measured bf16 peak when that bound is larger)
   cpu_baseline  the float64 CPU checker timed on a bounded sample of the same workload
+  parity    the device results of the timed workload compared with that checker run (same inputs,
+            verify seed 0, same sequences) under the rules of the parity tests
+
+The headline workload is the 405B-shaped head (largest single-GPU configuration); the other
+configurations are timed in the same run and summarised under `other_workloads`.
+`--record-traffic CSV...` does not measure anything: it reads ncu raw-page CSV exports and rewrites
+profiles/ncu_traffic.json (DRAM bytes per launch of the dominant kernels, with the hash of the
+kernel sources they were taken on).
 
 `--impl reference` times the CPU checker alone (rank 0 only).
 With --gpus N > 1 (launched under torchrun) every rank runs an independent replica: the path has
@@ -36,13 +44,60 @@ METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes (read + write) per verification call from the ncu captures summarised under profiles/
-# (dominant kernels of each workload); set an entry to None when its kernel changes.
-NCU_TRAFFIC_BYTES = {"cfg1-8B-head": 1.0593e9, "cfg2-70B-head": 2.1576e9, "cfg3-405B-head": 4.2244e9,
-                     "cfg3-405B-head-fp8": 2.1230e9,
-                     "cfg4-batched": 2.1495e9 + 2.1448e9,          # GEMM pass + second pass
-                     "cfg4-batched-fp8": 1.0666e9 + 1.0905e9}
 VARIANT_NAMES = {1: "simt", 2: "fused", 3: "batched"}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+KERNEL_SOURCES = ["jd_fused_sm100.cu", "jd_batched_sm100.cu", "jd_sm100_ptx.cuh", "jd_common.cuh"]
+
+
+def kernel_source_hash() -> str:
+    """sha256 over the sources of the tensor-core kernels: the DRAM counters are only quoted while
+    the kernels are the ones they were captured on."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2501_19309_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic_bytes(workload: str):
+    """DRAM bytes (read + write) per verification call from the ncu captures summarised under
+    profiles/, or None when there is no capture of the present kernels."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            t = json.load(f)
+    except (OSError, ValueError):
+        return None
+    if t.get("kernel_source_sha256_16") != kernel_source_hash():
+        return None
+    e = t.get("workloads", {}).get(workload)
+    return None if e is None else float(e["dram_bytes_per_call"])
+
+
+def record_traffic(csv_specs) -> None:
+    """csv_specs: 'workload=path[,path...]' items; every CSV is an `ncu --page raw --csv` export with
+    dram__bytes_read.sum / dram__bytes_write.sum columns. The bytes of the first captured launch of
+    each file are added up per workload (a workload whose call runs two kernels gives two files)."""
+    import csv
+    out = {"kernel_source_sha256_16": kernel_source_hash(), "workloads": {},
+           "note": "dram__bytes_read.sum + dram__bytes_write.sum of one launch of each dominant kernel"}
+    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    for spec in csv_specs:
+        name, paths = spec.split("=", 1)
+        total, kernels = 0.0, []
+        for path in paths.split(","):
+            with open(path, newline="") as f:
+                rows = [r for r in csv.reader(f) if r]
+            hdr = next(i for i, r in enumerate(rows) if "Kernel Name" in r)
+            cols, units, first = rows[hdr], rows[hdr + 1], rows[hdr + 2]
+            kernels.append(first[cols.index("Kernel Name")].split("(")[0])
+            for m in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+                i = cols.index(m)
+                total += float(first[i].replace(",", "")) * scale[units[i]]
+        out["workloads"][name] = {"dram_bytes_per_call": total, "kernels": kernels}
+    with open(TRAFFIC_FILE, "w") as f:
+        json.dump(out, f, indent=1, sort_keys=True)
+        f.write("\n")
 
 
 def load_peaks():
@@ -135,7 +190,7 @@ def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, 
         tf_peak, tf_sustained = 2 * tf_peak, 2 * tf_sustained
     t_bytes = bytes_alg / (peaks["hbm_gbs"] * 1e9)
     t_flops = flops / (tf_peak * 1e12)
-    traffic = NCU_TRAFFIC_BYTES.get(wl.name)
+    traffic = ncu_traffic_bytes(wl.name)
     if t_bytes >= t_flops:
         ach = bytes_alg / (kernel_ms * 1e-3) / 1e9
         return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -167,22 +222,56 @@ def cpu_threads() -> int:
         return os.cpu_count() or 1
 
 
-def time_oracle(inp: I.Inputs, steps: int, budget_s: float = 25.0) -> dict:
-    """The checker as it stands on a bounded sample: whole sequences b = 0, 1, ... of the workload."""
+def time_oracle(inp: I.Inputs, steps: int, budget_s: float = 25.0, extra_warmup: int = 0) -> dict:
+    """The checker as it stands on a bounded sample: whole sequences b = 0, 1, ... of the workload.
+    Step s uses verify seed s; "first" is the result of step 0 (kept for the parity check)."""
     wl = inp.wl
     t0 = time.perf_counter()
     oracle_step(inp, 0, [0])
     one = time.perf_counter() - t0
+    for _ in range(extra_warmup):          # untimed, on top of the sizing call above
+        oracle_step(inp, 0, [0])
     nseq = int(max(1, min(wl.B, budget_s / max(one, 1e-3) / max(steps, 1))))
     seqs = list(range(nseq))
+    first = None
     t0 = time.perf_counter()
     for s in range(steps):
-        oracle_step(inp, s, seqs)
+        r = oracle_step(inp, s, seqs)
+        first = first or r
     dt = time.perf_counter() - t0
     return {"value": nseq * wl.M * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
             "sample": "%d step(s) x %d of %d sequences (%d rows x V=%d x d=%d each), float64 numpy" %
                       (steps, nseq, wl.B, wl.M + 1, wl.V, wl.d),
-            "seconds": dt}
+            "seconds": dt, "first": first}
+
+
+def parity_of(wl: I.Workload, got: dict, ref) -> dict:
+    """Device outputs of verify seed 0 against the checker's result for the same inputs, under the
+    rules of the parity tests (tests/jd_testlib.py: tolerances, margin exemptions, CDF intervals)."""
+    tests_dir = os.path.join(ROOT, "tests")
+    if tests_dir not in sys.path:
+        sys.path.insert(0, tests_dir)
+    import jd_testlib as T
+    rep = T.Report()
+    try:
+        T.compare(got, ref, "judge_or_standard", wl.M, rep)
+        ok, why = True, None
+    except AssertionError as e:
+        ok, why = False, str(e)[:200]
+    out = {"sequences": rep.sequences, "ok": ok, "exempt": rep.exempt_accept + rep.exempt_judge,
+           "exempt_len": rep.exempt_len, "token_exact": rep.token_exact, "token_in_margin": rep.token_in_margin,
+           "max_rel_p": rep.max_rel_p, "max_rel_lse": rep.max_rel_lse, "max_abs_judge": rep.max_abs_judge}
+    if why:
+        out["failure"] = why
+    return out
+
+
+def config_of(wl: I.Workload, world: int) -> dict:
+    """The `config` object, identical in both arms."""
+    return {"workload": wl.name, "B": wl.B, "M": wl.M, "d": wl.d, "V": wl.V, "mode": "judge_or_standard",
+            "l2": "not flushed between calls: inputs larger than L2 (W is %.2f GB, L2 126 MB)" %
+                  (wl.V * wl.d * (1 if wl.dtype == "fp8" else 2) / 1e9),
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
 
 
 def run_reference(args, wl) -> None:
@@ -190,14 +279,19 @@ def run_reference(args, wl) -> None:
     if rank != 0:
         return
     inp = I.make_inputs(wl, 0)
-    steps = max(1, min(args.steps, 3))
-    for _ in range(min(args.warmup, 1)):
-        oracle_step(inp, 0, [0])
-    r = time_oracle(inp, steps, budget_s=60.0)
+    # K timed steps after W warm-up steps, as asked, each step a bounded sample (whole sequences) of
+    # the workload; only when K steps of even one sequence would run for more than ~5 minutes are
+    # they cut down, and the line says so
+    t0 = time.perf_counter()
+    oracle_step(inp, 0, [0])
+    one = time.perf_counter() - t0
+    steps = int(max(1, min(args.steps, 300.0 / max(one, 1e-3))))
+    warmup = int(max(2, min(args.warmup, 30.0 / max(one, 1e-3))))   # the call above + time_oracle's sizing call + ...
+    r = time_oracle(inp, steps, budget_s=max(60.0, one * steps), extra_warmup=warmup - 2)
     line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
-            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": r["seconds"] / steps * 1e3,
+            "steps": steps, "warmup": warmup, "ms_per_step": r["seconds"] / steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": wl.name, "B": wl.B, "M": wl.M, "d": wl.d, "V": wl.V},
+            "data": "synthetic", "config": config_of(wl, 1),
             "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
             "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -288,6 +382,9 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
         step(i)
         accepted.append(out["accept_len"].cpu().numpy().astype(np.float64))
     accepted = np.stack(accepted)
+    step(0)                                   # verify seed 0 once more: the outputs the parity check reads
+    torch.cuda.synchronize(device)
+    out0 = {k: v.detach().cpu().numpy().copy() for k, v in out.items()}
 
     # read-only streaming ceiling of this device: the library's probe over the same W
     sink = torch.zeros(1, dtype=torch.int32, device=device)
@@ -325,7 +422,7 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     res = dict(total_ms=total_ms, median_ms=statistics.median(per), min_ms=min(per), mean_ms=total_ms / K,
                variant=variant, launches=launches, clocks=clocks, e2e_s=e2e_s, e2e_steps=Ke, h2d=h2d, d2h=d2h,
                mean_accept=float(accepted.mean()), emitted_per_call=float((accepted + 1).sum(axis=1).mean()),
-               stream_gbs=stream_gbs, graph_ms=graph_ms, inp=inp)
+               stream_gbs=stream_gbs, graph_ms=graph_ms, inp=inp, out0=out0)
     del W, H, dl
     torch.cuda.empty_cache()
     return res
@@ -337,14 +434,20 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, help="workload id of the headline line (1..4)")
-    ap.add_argument("--others", default="2,3,4,3f,4f", help="comma list of further workloads summarised in the same "
+    ap.add_argument("--config", type=int, default=3, help="workload id of the headline line (1..4); default: the "
+                    "405B-shaped head, the largest single-GPU configuration")
+    ap.add_argument("--others", default="2,1,4,3f,4f", help="comma list of further workloads summarised in the same "
                     "line; a trailing f = the same shape with an FP8 E4M3 head")
+    ap.add_argument("--record-traffic", nargs="+", metavar="WORKLOAD=CSV[,CSV]", help="rewrite profiles/ncu_traffic.json "
+                    "from ncu raw-page CSV exports and exit")
     ap.add_argument("--fp8", action="store_true", help="headline workload with an FP8 E4M3 head")
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
     args = ap.parse_args()
+    if args.record_traffic:
+        record_traffic(args.record_traffic)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = I.CONFIGS[args.config]
     if args.fp8:
@@ -392,6 +495,12 @@ def main() -> None:
             small.steps = max(50, min(args.steps, 300))
             small.e2e_steps = 10
             r = measure_workload(owl, small, torch, jd, device, data_seed=0, sample_clocks=True)
+            oparity = None
+            if not args.no_cpu_baseline:      # a few seconds of the checker on the first sequences
+                oparity = parity_of(owl, r["out0"], time_oracle(r["inp"], 1, budget_s=5.0)["first"])
+            e2e_note = None
+            if owl.B * owl.M * owl.V * 4 > 100e6:
+                e2e_note = ("%.0f MB of fp32 draft logits cross PCIe per host-buffer call" % (owl.B * owl.M * owl.V * 4 / 1e6))
             others[owl.name] = {
                 "B": owl.B, "M": owl.M, "d": owl.d, "V": owl.V, "ms_per_step": r["mean_ms"],
                 "median_ms": r["median_ms"], "value": owl.B * owl.M / (r["mean_ms"] * 1e-3), "unit": UNIT,
@@ -400,24 +509,25 @@ def main() -> None:
                 "clocks": r["clocks"],
                 "graph_replay_ms_per_step": r["graph_ms"],
                 "emitted_tokens_per_s": r["emitted_per_call"] / (r["mean_ms"] * 1e-3),
-                "e2e_value": owl.B * owl.M * r["e2e_steps"] / r["e2e_s"],
+                "e2e": {"value": owl.B * owl.M * r["e2e_steps"] / r["e2e_s"], "unit": UNIT,
+                        "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"], "steps": r["e2e_steps"],
+                        "note": e2e_note},
+                "parity": oparity,
                 "roofline": roofline_of(owl, peaks, r["mean_ms"], sustained=r["mean_ms"] * small.steps > 1000, which=which,
                                         stream_gbs=r["stream_gbs"])}
 
     if rank == 0:
-        cpu = None
+        cpu, parity = None, None
         if not args.no_cpu_baseline:
             c = time_oracle(res["inp"], 1)
             cpu = {k: c[k] for k in ("value", "unit", "cores", "kind", "sample")}
+            parity = parity_of(wl, res["out0"], c["first"])
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "fp8" if wl.dtype == "fp8" else "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "M": wl.M, "d": wl.d, "V": wl.V, "mode": "judge_or_standard",
-                       "variant": VARIANT_NAMES.get(res["variant"], "?"),
-                       "l2": "inputs larger than L2: W (%.2f GB) streams from HBM every call" % (wl.V * wl.d * 2 / 1e9),
-                       "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "mean_accept_len": res["mean_accept"]},
+            "config": config_of(wl, world),
+            "variant": VARIANT_NAMES.get(res["variant"], "?"), "mean_accept_len": res["mean_accept"],
             "calls_per_s": world * K / (total_ms * 1e-3),
             "median_ms_per_step": res["median_ms"],
             "best_ms_per_step": res["min_ms"],
@@ -430,6 +540,7 @@ def main() -> None:
             "roofline": roofline_of(wl, peaks, res["mean_ms"], sustained=total_ms > 1000, which=which,
                                     stream_gbs=res["stream_gbs"]),
             "cpu_baseline": cpu,
+            "parity": parity,
             "other_workloads": others,
         }
         print(json.dumps(line), flush=True)

@@ -60,7 +60,7 @@ typedef enum { JD_MODE_STANDARD = 0, JD_MODE_JUDGE = 1, JD_MODE_JUDGE_OR_STANDAR
 /* Distribution of the token drawn at the first rejected slot a < M.
  * RESIDUAL: normalised max(0, p_a - q_a), the form under which the standard test is lossless;
  *           an identically zero residual falls back to p_a.
- * TARGET_P: p_a itself, the literal wording of Sec. 3.1 ("sample a correct token from p_i").
+ * TARGET_P: p_a itself, which is how Sec. 3.1 words the correction when read literally.
  * After a fully accepted block the token always comes from p_M. */
 typedef enum { JD_RESAMPLE_RESIDUAL = 0, JD_RESAMPLE_TARGET_P = 1 } jd_resample_t;
 
@@ -74,10 +74,10 @@ typedef enum { JD_RESAMPLE_RESIDUAL = 0, JD_RESAMPLE_TARGET_P = 1 } jd_resample_
  *           only feed the q_draft output. */
 typedef enum { JD_RULE_SAMPLING = 0, JD_RULE_TOPK = 1 } jd_rule_t;
 
-/* Normalisation applied to the rows of H in front of the LM head. The paper's judge reads the last
- * embedding "before the RMS normalization and the LM head" (Sec. 4.1): with JD_NORM_RMS the logits
- * are W . (H[b,j] / sqrt(mean_k H[b,j,k]^2 + rms_eps)) while the judge dot product still uses
- * H[b,j+1] as given. The norm's gain vector is expected folded into W. */
+/* Normalisation applied to the rows of H in front of the LM head. The paper's judge takes the last
+ * embedding ahead of the model's final RMS norm and LM head (Sec. 4.1 "Model design and training"):
+ * with JD_NORM_RMS the logits are W . (H[b,j] / sqrt(mean_k H[b,j,k]^2 + rms_eps)) while the judge
+ * dot product still uses H[b,j+1] as given. The norm's gain vector is expected folded into W. */
 typedef enum { JD_NORM_NONE = 0, JD_NORM_RMS = 1 } jd_norm_t;
 
 /* Kernel family used by jd_verify. AUTO picks the fastest one that supports the shape. */
@@ -110,7 +110,9 @@ typedef struct {
   const void* H;               /* [B, M+1, d] embeddings, dtype of the handle (bf16 for an FP8 head),
                                   16-byte aligned */
   const int32_t* draft_tokens; /* [B, M] drafted token ids x_j in [0, V) */
-  const float* draft_logits;   /* [B, M, V] draft-model logits; q_j = softmax at temperature 1 */
+  const float* draft_logits;   /* [B, M, V] draft-model logits; q_j = softmax at temperature 1. 4-byte aligned
+                                  like every int32 / float array here; a 16-byte aligned base with V % 4 == 0
+                                  lets the kernels use 16-byte loads, anything else takes 4-byte loads */
   float tau;                   /* judge threshold in [0, 1]; accept iff score > tau (strict) */
   uint64_t seed;               /* Philox key */
   int32_t mode;                /* jd_mode_t */
@@ -130,7 +132,9 @@ typedef struct {
   uint8_t* masks;              /* [B, M] bit0 = standard test passed, bit1 = judge test passed */
   float* row_max;              /* [B, M+1] max_v L[b,j,v] */
   float* row_lse;              /* [B, M+1] log sum_v exp L[b,j,v] */
-  float* logits_debug;         /* [B, M+1, V] the logits; tests only, SIMT variant only */
+  float* logits_debug;         /* [B, M+1, V] the logits as the softmax sees them (normalisation and FP8
+                                  scales applied); tests only: every variant honours it, at the price of
+                                  writing R x V floats */
 } jd_verify_args_t;
 
 /* Library version, major*10000 + minor*100 + patch. */
@@ -163,8 +167,11 @@ jd_status_t jd_set_head(jd_handle_t h, const void* W, const void* w_judge, float
  * of H the same way on the device, s_r = max_k |H[r,k]| / 448 and h8 = e4m3(H[r,k] * 448 / max_k |H[r,k]|)
  * rounded to nearest even, and the tensor cores multiply FP8 by FP8 with fp32 accumulation:
  * L[r,v] = w_scale[v] * s_r * sum_k e4m3(W8[v,k]) * h8[r,k]. The judge still reads the bf16 rows.
- * w_judge [d] is bf16. Pointers are borrowed like those of jd_set_head. Requires d % 128 == 0 for
- * the tensor-core variant (the CUDA-core variant takes any d); the batched variant has no FP8 form. */
+ * h8 is the E4M3 value nearest to that quotient, ties to the even mantissa (the device computes
+ * H * 448 in float32, exactly, and divides with one rounding, which yields the same codes as the
+ * exact quotient for bf16 rows). w_judge [d] is bf16. Pointers are borrowed like those of
+ * jd_set_head. The fused and the batched tensor-core variants need d % 128 == 0; the CUDA-core
+ * variant takes any d. */
 jd_status_t jd_set_head_fp8(jd_handle_t h, const void* W8, const float* w_scale, const void* w_judge,
                             float b_judge);
 
@@ -215,6 +222,19 @@ jd_status_t jd_stream_read_probe(const void* data, size_t bytes, uint32_t* out, 
 jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* slot,
                                const int32_t* stream, int32_t n, float* out, void* cuda_stream);
 
+/* Test helper for the FP8 head: quantises `rows` bf16 rows of width d (device pointer, 16-byte
+ * aligned) exactly as jd_verify does for a JD_DTYPE_FP8_E4M3 handle and writes the E4M3 codes
+ * [rows, d] (device pointer, 16-byte aligned) and the per-row scales [rows] (float32). Asynchronous
+ * on the stream; uses the current device. */
+jd_status_t jd_quantize_rows_e4m3(const void* H, int32_t rows, int32_t d, uint8_t* codes, float* scale,
+                                  void* cuda_stream);
+
+/* Test helper (the paper has no counterpart): the handle's workspace regions are separated by guard
+ * blocks of a fixed byte pattern that no kernel may touch. Synchronises the device and sets
+ * *damaged to the number of guard blocks whose pattern is no longer intact (0 = no kernel wrote
+ * past the end of a region). */
+jd_status_t jd_check_workspace_guards(jd_handle_t h, int32_t* damaged);
+
 /* Handle-free form of jd_verify for callers that must not allocate device memory when they
  * verify: servers whose own pool already owns the whole device, decode loops that cannot afford
  * the synchronisation an allocation implies, code barred from allocating after start-up.
@@ -230,7 +250,9 @@ jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* s
  *   device_status            : optional device pointer to one uint32 that receives the call's
  *                              device status (JD_OK, JD_ERR_TIMEOUT, JD_ERR_BAD_TOKEN); NULL to skip
  * The call uses the CURRENT device. Its first call on a device looks up the array's device
- * address and the SM count; make that first call outside any stream capture. All calls on a
+ * address and the SM count and loads every instantiation of the kernel (so that no later call has
+ * to load code); make that first call outside any stream capture. First calls from several host
+ * threads are serialised by a lock. All calls on a
  * device share the one array, which keeps the previous call's contents (the words that must
  * start at zero are cleared on the stream each time): calls that overlap on the GPU, from any
  * stream or thread, race with each other, so order them. Asynchronous on `cuda_stream`. */

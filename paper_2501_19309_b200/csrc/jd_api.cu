@@ -11,6 +11,10 @@
 
 using namespace jd;
 
+constexpr int kMaxGuards = 48;
+constexpr size_t kGuardBytes = 256;
+constexpr unsigned char kGuardByte = 0xC5;
+
 struct jd_handle_s {
   jd_config_t cfg;
   int num_sms;
@@ -41,6 +45,15 @@ struct jd_handle_s {
   unsigned dl_epoch;
   cudaEvent_t dl_event;    // recorded on the side stream after that copy
   bool dl_in_flight;       // true only inside jd_verify_host, between enqueueing the copy and jd_verify
+  // tensor map of the caller's H, kept from the previous call (decode loops reuse their buffers)
+  CUtensorMap tm_h_cached;
+  const void* tm_h_base;
+  uint64_t tm_h_rows;
+  uint32_t tm_h_box;
+  bool tm_h_bytes;
+  // guard blocks between the regions of the workspace (offsets into ws_base)
+  int n_guards;
+  size_t guard_off[kMaxGuards];
 };
 
 namespace {
@@ -105,15 +118,21 @@ bool config_ok(const jd_config_t* c) {
   return true;
 }
 
-// Carves the workspace; with base == nullptr only measures it.
-size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
+// Carves the workspace; with base == nullptr only measures it. Every region is followed by a guard
+// block of kGuardBytes that no kernel may write; guard_off (optional) receives their offsets.
+size_t carve(const jd_config_t& c, char* base, Workspace* ws, size_t* guard_off = nullptr, int* n_guards = nullptr,
+             unsigned** dl_flag = nullptr) {
   const size_t maxB = c.max_B, maxR = (size_t)c.max_B * (c.max_M + 1), maxBM = (size_t)c.max_B * c.max_M;
   const size_t np = std::max<size_t>((c.V + kVocabTile - 1) / kVocabTile, kMaxCtas);
   const size_t nq = std::max<size_t>((c.V + 8191) / 8192, kMaxCtas);
   size_t off = 0;
+  int ng = 0;
   auto take = [&](size_t bytes) {
     char* p = base ? base + off : nullptr;
     off += align_up(bytes, 256);
+    if (guard_off && ng < kMaxGuards) guard_off[ng] = off;
+    ++ng;
+    off += kGuardBytes;
     return p;
   };
   Workspace w;
@@ -143,12 +162,14 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
   w.cnt = (int*)take(maxR * 4);
   w.argidx = (int*)take(maxR * 4);
   w.part_idx = (int*)take(maxR * np * 4);
-  w.status = (unsigned*)take(256);
-  w.barrier = (unsigned*)take(256);
-  take(256);   // word 0: arrival flag of a host-buffer call's draft logits; outside the per-call memset
+  w.status = (unsigned*)take(512);   // status word and, 256 bytes on, the barrier counters: one memset per call
+  w.barrier = w.status ? w.status + 64 : nullptr;
+  char* flag = take(256);   // word 0: arrival flag of a host-buffer call's draft logits; outside the per-call memset
+  if (dl_flag) *dl_flag = (unsigned*)flag;
   w.np_cap = (int)np;
   w.nq_cap = (int)nq;
   if (ws) *ws = w;
+  if (n_guards) *n_guards = ng < kMaxGuards ? ng : kMaxGuards;
   return off;
 }
 
@@ -156,6 +177,19 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws) {
 size_t elem_size(int dtype) { return dtype == JD_DTYPE_F32 ? 4 : 2; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+bool configure_kernels() { return fused_configure() && batched_configure(); }
+
+// The tensor map of the caller's H: re-encoded only when the pointer, the row count or the box changes.
+const CUtensorMap* h_tensor_map(jd_handle_t h, const void* base, uint64_t rows, uint32_t box_rows, bool bytes) {
+  if (h->tm_h_base != base || h->tm_h_rows != rows || h->tm_h_box != box_rows || h->tm_h_bytes != bytes) {
+    h->tm_h_base = nullptr;
+    if (!make_tensor_map(&h->tm_h_cached, base, rows, (uint64_t)h->cfg.d, box_rows, bytes)) return nullptr;
+    h->tm_h_base = base; h->tm_h_rows = rows; h->tm_h_box = box_rows; h->tm_h_bytes = bytes;
+  }
+  return &h->tm_h_cached;
+}
 
 jd_status_t validate(jd_handle_t h, const jd_verify_args_t* a) {
   if (!h || !a) return JD_ERR_INVALID_ARG;
@@ -171,6 +205,11 @@ jd_status_t validate(jd_handle_t h, const jd_verify_args_t* a) {
   if (a->rule == JD_RULE_TOPK && a->top_k < 1) return JD_ERR_INVALID_ARG;
   if (a->norm != JD_NORM_NONE && a->norm != JD_NORM_RMS) return JD_ERR_INVALID_ARG;
   if (a->norm == JD_NORM_RMS && !(a->rms_eps >= 0.f)) return JD_ERR_INVALID_ARG;
+  // natural alignment of every 4-byte array (device or host); H is checked by the device entry point
+  if (!aligned4(a->draft_tokens) || !aligned4(a->draft_logits) || !aligned4(a->accept_len) || !aligned4(a->next_token) ||
+      !aligned4(a->judge_scores) || !aligned4(a->p_draft) || !aligned4(a->q_draft) || !aligned4(a->row_max) ||
+      !aligned4(a->row_lse) || !aligned4(a->logits_debug))
+    return JD_ERR_INVALID_ARG;
   return JD_OK;
 }
 
@@ -218,8 +257,12 @@ jd_status_t jd_create(jd_handle_t* out, const jd_config_t* cfg) {
     delete h;
     return JD_ERR_ALLOC;
   }
-  carve(*cfg, (char*)h->ws_base, &h->ws);
-  if (cudaMemset(h->ws_base, 0, h->ws_bytes) != cudaSuccess) {
+  carve(*cfg, (char*)h->ws_base, &h->ws, h->guard_off, &h->n_guards, &h->dl_flag);
+  bool filled = cudaMemset(h->ws_base, 0, h->ws_bytes) == cudaSuccess;
+  for (int g = 0; g < h->n_guards && filled; ++g)
+    filled = cudaMemset((char*)h->ws_base + h->guard_off[g], kGuardByte, kGuardBytes) == cudaSuccess;
+  if (!filled || !configure_kernels()) {
+    cudaGetLastError();
     cudaFree(h->ws_base);
     delete h;
     return JD_ERR_CUDA;
@@ -234,7 +277,6 @@ jd_status_t jd_create(jd_handle_t* out, const jd_config_t* cfg) {
     if (h->side.join) cudaEventDestroy(h->side.join);
     h->side = SideStream{};
   }
-  h->dl_flag = h->ws.barrier + 64;
   if (h->side.stream && cudaEventCreateWithFlags(&h->dl_event, cudaEventDisableTiming) != cudaSuccess) {
     cudaGetLastError();
     h->dl_event = nullptr;
@@ -312,6 +354,10 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   cp.judge_scores = a->judge_scores; cp.p_draft = a->p_draft;
   cp.q_draft = a->q_draft; cp.masks = a->masks;
   cp.row_max_out = a->row_max; cp.row_lse_out = a->row_lse;
+  cp.logits_debug = a->logits_debug;
+  // 16-byte loads of the draft logits need every row on a 16-byte boundary; a 4-byte-aligned view
+  // (a slice of a larger buffer) takes the kernels' 4-byte path instead
+  cp.dl_vec4 = (c.V % 4 == 0 && aligned16(a->draft_logits)) ? 1 : 0;
 
   FusedPlan plan;
   const bool fused_ok = h->tm_w_ok && fused_supported(c.dtype, R, c.d, c.V, h->num_sms, &plan);
@@ -319,13 +365,12 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   const bool batched_ok = h->tm_w_ok && batched_supported(c.dtype, a->B, c.d, c.V, h->num_sms);
   int variant = a->variant;
   if (variant == JD_VARIANT_AUTO) {
-    if (a->logits_debug) variant = JD_VARIANT_SIMT;
-    else if (fused_ok) variant = JD_VARIANT_FUSED;
+    if (fused_ok) variant = JD_VARIANT_FUSED;
     else if (batched_ok) variant = JD_VARIANT_BATCHED;
     else variant = JD_VARIANT_SIMT;
   }
-  if (variant == JD_VARIANT_FUSED && (!fused_ok || a->logits_debug)) return JD_ERR_UNSUPPORTED;
-  if (variant == JD_VARIANT_BATCHED && (!batched_ok || a->logits_debug)) return JD_ERR_UNSUPPORTED;
+  if (variant == JD_VARIANT_FUSED && !fused_ok) return JD_ERR_UNSUPPORTED;
+  if (variant == JD_VARIANT_BATCHED && !batched_ok) return JD_ERR_UNSUPPORTED;
 
   if (cudaSetDevice(c.device) != cudaSuccess) return JD_ERR_CUDA;
   // status word and the grid-barrier counters behind it start every call at zero
@@ -351,16 +396,18 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
     if (variant == JD_VARIANT_SIMT && cudaStreamWaitEvent(st, h->dl_event, 0) != cudaSuccess) return JD_ERR_CUDA;
   }
   if (variant == JD_VARIANT_SIMT) {
-    launches += run_simt(cp, h->ws, h->W, h->w_scale, h->w_judge, a->H, c.dtype, a->logits_debug, st);
+    launches += run_simt(cp, h->ws, h->W, h->w_scale, h->w_judge, a->H, c.dtype, st);
   } else if (variant == JD_VARIANT_BATCHED) {
     // second pass: the selected rows go through the fused kernel, a chunk of sequences per launch
     const int chunk = second_pass_chunk(a->B), tail = a->B % chunk;
     FusedPlan plan2, plan3;
     if (!fused_supported(c.dtype, chunk, c.d, c.V, h->num_sms, &plan2)) return JD_ERR_UNSUPPORTED;
     if (tail && !fused_supported(c.dtype, tail, c.d, c.V, h->num_sms, &plan3)) return JD_ERR_UNSUPPORTED;
-    CUtensorMap tm_h, tm_hsel, tm_hsel_tail;
-    if (!make_tensor_map(&tm_h, fp8 ? (const void*)h->ws.h8 : a->H, (uint64_t)R, (uint64_t)c.d, 128, fp8) ||
-        !make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)chunk, (uint64_t)c.d, (uint32_t)plan2.n_pad, fp8))
+    CUtensorMap tm_hsel, tm_hsel_tail;
+    const CUtensorMap* tm_hp = h_tensor_map(h, fp8 ? (const void*)h->ws.h8 : a->H, (uint64_t)R, 128, fp8);
+    if (!tm_hp) return JD_ERR_CUDA;
+    const CUtensorMap& tm_h = *tm_hp;
+    if (!make_tensor_map(&tm_hsel, h->ws.h_sel, (uint64_t)chunk, (uint64_t)c.d, (uint32_t)plan2.n_pad, fp8))
       return JD_ERR_CUDA;
     tm_hsel_tail = tm_hsel;
     if (tail && !make_tensor_map(&tm_hsel_tail, h->ws.h_sel, (uint64_t)tail, (uint64_t)c.d, (uint32_t)plan3.n_pad, fp8))
@@ -371,11 +418,10 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
     if (n < 0) return JD_ERR_CUDA;
     launches += n;
   } else {
-    CUtensorMap tm_h;
-    if (!make_tensor_map(&tm_h, fp8 ? (const void*)h->ws.h8 : a->H, (uint64_t)R, (uint64_t)c.d, (uint32_t)plan.n_pad, fp8))
-      return JD_ERR_CUDA;
+    const CUtensorMap* tm_hp = h_tensor_map(h, fp8 ? (const void*)h->ws.h8 : a->H, (uint64_t)R, (uint32_t)plan.n_pad, fp8);
+    if (!tm_hp) return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
-    const int n = run_fused(cp, h->ws, h->tm_w, tm_h, a->H, h->w_judge, plan, st, &err, false, fp8 ? h->w_scale : nullptr,
+    const int n = run_fused(cp, h->ws, h->tm_w, *tm_hp, a->H, h->w_judge, plan, st, &err, false, fp8 ? h->w_scale : nullptr,
                             h->dl_in_flight ? h->dl_flag : nullptr, h->dl_epoch);
     if (n < 0) return JD_ERR_CUDA;
     launches += n;
@@ -519,6 +565,35 @@ jd_status_t jd_philox_uniforms(uint64_t seed, const int32_t* b, const int32_t* s
   if (n == 0) return JD_OK;
   launch_philox_uniforms(seed, b, slot, stream, n, out, (cudaStream_t)cuda_stream);
   return cudaGetLastError() == cudaSuccess ? JD_OK : JD_ERR_CUDA;
+}
+
+jd_status_t jd_quantize_rows_e4m3(const void* H, int32_t rows, int32_t d, uint8_t* codes, float* scale,
+                                  void* cuda_stream) {
+  if (!H || !codes || !scale || rows < 1 || d < 1) return JD_ERR_INVALID_ARG;
+  if (!aligned16(H) || !aligned16(codes) || !aligned4(scale)) return JD_ERR_INVALID_ARG;
+  CallParams cp = {};
+  cp.B = rows; cp.M = 0; cp.d = d;   // rows x 1 "sequences": the launcher quantises B * (M + 1) rows
+  Workspace ws = {};
+  ws.h8 = codes;
+  ws.h_scale = scale;
+  launch_quantize_rows(cp, ws, H, (cudaStream_t)cuda_stream);
+  return cudaGetLastError() == cudaSuccess ? JD_OK : JD_ERR_CUDA;
+}
+
+jd_status_t jd_check_workspace_guards(jd_handle_t h, int32_t* damaged) {
+  if (!h || !damaged) return JD_ERR_INVALID_ARG;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return JD_ERR_CUDA;
+  if (cudaDeviceSynchronize() != cudaSuccess) return JD_ERR_CUDA;
+  unsigned char block[kGuardBytes];
+  int bad = 0;
+  for (int g = 0; g < h->n_guards; ++g) {
+    if (cudaMemcpy(block, (const char*)h->ws_base + h->guard_off[g], kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return JD_ERR_CUDA;
+    for (size_t i = 0; i < kGuardBytes; ++i)
+      if (block[i] != kGuardByte) { ++bad; break; }
+  }
+  *damaged = bad;
+  return JD_OK;
 }
 
 }  // extern "C"

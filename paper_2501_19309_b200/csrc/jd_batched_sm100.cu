@@ -196,6 +196,11 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           for (int k = 0; k < 32; ++k) v[k] *= sc;
         }
         const int nvalid = cp.V - (v0 + c0);   // columns of this chunk that exist (>= 32 except at the tail)
+        if (!kCount && cp.logits_debug != nullptr && row < R) {   // test-only copy of the logits
+          float* o = cp.logits_debug + (size_t)row * cp.V + v0 + c0;
+#pragma unroll
+          for (int k = 0; k < 32; ++k) if (k < nvalid) o[k] = v[k];
+        }
         if (nvalid < 32) {
 #pragma unroll
           for (int k = 0; k < 32; ++k) if (k >= nvalid) v[k] = -INFINITY;
@@ -285,6 +290,13 @@ static int grid_of(int R, int np, int num_sms) {
   return std::min(num_sms, ((R + kTileM - 1) / kTileM) * np);
 }
 
+bool batched_configure() {
+  return cudaFuncSetAttribute(gemm_stats_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess &&
+         cudaFuncSetAttribute(gemm_stats_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess &&
+         cudaFuncSetAttribute(gemm_stats_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess &&
+         cudaFuncSetAttribute(gemm_stats_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess;
+}
+
 bool batched_supported(int dtype, int B, int d, int V, int num_sms) {
   if (dtype == JD_DTYPE_BF16) { if (d % kTileK != 0 || d < kTileK) return false; }
   else if (dtype == JD_DTYPE_FP8_E4M3) { if (d % (2 * kTileK) != 0 || d < 2 * kTileK) return false; }
@@ -309,8 +321,6 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
   auto gemm = [&](bool count) {
     auto kern = fp8 ? (count ? gemm_stats_kernel<true, true> : gemm_stats_kernel<false, true>)
                     : (count ? gemm_stats_kernel<true, false> : gemm_stats_kernel<false, false>);
-    *err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (*err != cudaSuccess) return false;
     kern<<<grid_of(R, np, num_sms), kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np, w_scale_fp8);
     return true;
   };
@@ -343,6 +353,7 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
     const int nc = std::min(chunk, cp.B - off);
     // this chunk's view of the call: sequences off .. off + nc - 1 become 0 .. nc - 1
     CallParams cc = cp;
+    cc.logits_debug = nullptr;   // the second pass recomputes selected rows only
     cc.B = nc;
     cc.next_token = cp.next_token + off;
     Workspace wc = ws;

@@ -143,6 +143,9 @@ struct CallParams {
   uint8_t* masks;
   float* row_max_out;
   float* row_lse_out;
+  float* logits_debug;   // [B, M+1, V] test-only copy of the logits (null in production)
+  int dl_vec4;           // 1: every draft-logit row starts on a 16-byte boundary (V % 4 == 0 and an aligned base),
+                         //    so the draft statistics may use 16-byte loads; 0: 4-byte loads only
 };
 
 // Decision step for one sequence b, executed by one warp (Eq. 4, Sec. 4.1 "Inference"):

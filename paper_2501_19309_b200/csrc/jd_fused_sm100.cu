@@ -158,6 +158,29 @@ __device__ __forceinline__ void load_cols8(int i0, int T, int r, int n_ovf, int 
   for (int u = 0; u < 8; ++u) out[u] = __uint_as_float(raw[u]) * (f * swt[min(i0 + u, 7) * kVocabTile + tid]);
 }
 
+// Test-only: copies the logits of this CTA's vocabulary slice to out[row, v] exactly as the
+// statistics passes read them (normalisation factors and FP8 scales applied). Called by the four
+// epilogue warps together; kept out of line so that the kernel's register allocation ignores it.
+template <int N_PAD>
+__device__ __noinline__ void dump_logits(float* __restrict__ out, int T, int t0, int R, int V, int n_ovf, int ts,
+                                         uint32_t tmem_lane_base, const float* ovf, int tid, const float* sc,
+                                         const float* swt) {
+  for (int i0 = 0; i0 < T; i0 += 2) {
+    const int vg0 = (t0 + i0) * kVocabTile + tid, vg1 = vg0 + kVocabTile;
+    const bool val0 = vg0 < V, val1 = (i0 + 1 < T) && vg1 < V;
+    for (int c0 = 0; c0 < N_PAD; c0 += 16) {
+      float v0[16], v1[16];
+      load_chunk2<N_PAD>(i0, T, c0, n_ovf, ts, tmem_lane_base, ovf, tid, sc, swt, v0, v1);
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        const int r = c0 + k;
+        if (r < R && val0) out[(size_t)r * V + vg0] = v0[k];
+        if (r < R && val1) out[(size_t)r * V + vg1] = v1[k];
+      }
+    }
+  }
+}
+
 // kFp8 is a template parameter, not a runtime flag: a kernel whose MMA loop can reach both
 // tcgen05.mma kinds ran its bf16 main loop 40 % slower.
 template <int N_PAD, bool kFp8>
@@ -366,7 +389,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       epi_sync();
     }
     const int v_lo = t0 * kVocabTile, v_hi = min(V, (t0 + T) * kVocabTile);
-    const bool vec4 = (V % 4) == 0;   // rows are 16-byte aligned only then
+    const bool vec4 = cp.dl_vec4 != 0;   // rows start on 16-byte boundaries only then
     for (int bm = warp; bm < (fp.sample_only ? 0 : BM); bm += 4) {
       const float* row = cp.draft_logits + (size_t)bm * V;
       float m = -INFINITY, s = 0.f;
@@ -610,6 +633,8 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       epi_sync();
     }
     if (!fp.sample_only) {
+    if (ok && cp.logits_debug != nullptr)
+      dump_logits<N_PAD>(cp.logits_debug, T, t0, R, V, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0]);
     __threadfence();
     epi_sync();
 
@@ -1018,9 +1043,7 @@ template <int N_PAD, bool kFp8>
 cudaError_t launch_fused(const CUtensorMap& tmW, const CUtensorMap& tmH, const CallParams& cp, const Workspace& ws,
                          const void* H, const void* wj, const float* w_scale, const FusedParams& fp,
                          const FusedPlan& plan, cudaStream_t st) {
-  auto kern = fused_verify_kernel<N_PAD, kFp8>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
-  if (e != cudaSuccess) return e;
+  auto kern = fused_verify_kernel<N_PAD, kFp8>;   // its shared-memory limit was raised by fused_configure()
   const __nv_bfloat16* Hp = (const __nv_bfloat16*)H;
   const __nv_bfloat16* wp = (const __nv_bfloat16*)wj;
   void* args[] = {(void*)&tmW, (void*)&tmH, (void*)&cp, (void*)&ws, (void*)&Hp, (void*)&wp, (void*)&w_scale, (void*)&fp};
@@ -1044,6 +1067,21 @@ void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st) 
   timeout_probe_kernel<<<2, 32, 0, st>>>(ws, limit);
 }
 
+namespace {
+template <int N_PAD>
+bool configure_pair() {
+  return cudaFuncSetAttribute(fused_verify_kernel<N_PAD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kMaxDynamicSmem) == cudaSuccess &&
+         cudaFuncSetAttribute(fused_verify_kernel<N_PAD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kMaxDynamicSmem) == cudaSuccess;
+}
+}  // namespace
+
+bool fused_configure() {
+  return configure_pair<16>() && configure_pair<32>() && configure_pair<48>() && configure_pair<64>() &&
+         configure_pair<80>() && configure_pair<96>();
+}
+
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan) {
   const bool fp8 = dtype == JD_DTYPE_FP8_E4M3;
   if (dtype != JD_DTYPE_BF16 && !fp8) return false;
@@ -1064,7 +1102,7 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
   if (fp8 && max_tiles > 8) return false;  // the per-tile vocabulary scales are kept for eight tiles
   const size_t base_fixed = 1024 /*alignment slack*/ + kMiscBytes + (size_t)n_ovf * kVocabTile * n_pad * 4;
   const size_t h_stage = (size_t)n_pad * 128;
-  const size_t budget = 227 * 1024;
+  const size_t budget = kMaxDynamicSmem;
   size_t fixed = base_fixed + kMinHStages * h_stage;
   if (fixed + 3 * (size_t)kWStageBytes > budget) return false;   // at least a three-deep W ring
   int stages = (int)((budget - fixed) / kWStageBytes);

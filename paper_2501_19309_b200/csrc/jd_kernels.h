@@ -9,8 +9,7 @@ namespace jd {
 
 // CUDA-core pipeline (jd_simt.cu). Each returns after enqueueing on `st`.
 int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const float* w_scale, const void* w_judge,
-             const void* H, int dtype,
-             float* logits_debug, cudaStream_t st);
+             const void* H, int dtype, cudaStream_t st);
 int launch_q_stats(const CallParams& cp, const Workspace& ws, cudaStream_t st);   // returns partials per draft row
 void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, const void* w, int dtype, cudaStream_t st);
 void launch_quantize_rows(const CallParams& cp, const Workspace& ws, const void* H_bf16, cudaStream_t st);
@@ -33,6 +32,12 @@ struct FusedPlan {
   int stages;         // W ring depth
   int h_stages;       // H ring depth
 };
+// Raises the dynamic shared-memory limit of every instantiation of a family's kernels on the CURRENT
+// device (which also loads them), once per device, ahead of the first launch: the launch paths set no
+// function attributes themselves.
+constexpr int kMaxDynamicSmem = 227 * 1024;
+bool fused_configure();
+bool batched_configure();
 void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st);
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan);
 // Returns the number of kernels launched, or -1 with *err set. dl_flag (optional): a device word

@@ -171,8 +171,8 @@ __global__ void __launch_bounds__(256) q_stats_kernel(CallParams cp, Workspace w
   const float* row = cp.draft_logits + (size_t)bm * V;
   const int lo = chunk * kQChunk, hi = min(V, lo + kQChunk);
   float m = -INFINITY, s = 0.f;
-  if ((V & 3) == 0) {
-    // rows are 16-byte aligned: every thread fetches its eight float4 of the chunk before any
+  if (cp.dl_vec4) {
+    // rows start on 16-byte boundaries: every thread fetches its eight float4 of the chunk before any
     // arithmetic, then takes the maximum and the sum of exponentials from registers
     float4 x[8];
 #pragma unroll
@@ -212,7 +212,15 @@ __global__ void __launch_bounds__(256) q_stats_kernel(CallParams cp, Workspace w
 }
 
 // FP8 head: quantises every row of H to E4M3 with one scale per row, s = amax / 448 and
-// code = e4m3(h * (448 / amax)), round to nearest even, saturating; all in float32.
+// code = e4m3(h * 448 / amax), round to nearest even, saturating. h * 448 is exact in float32 for a
+// bf16 h (8 + 3 significant bits) and the division rounds once, to 24 bits; a quotient of two bf16
+// values that is not itself a half-way point of the E4M3 grid stays at least 2^-14 (relative) away
+// from one, so the second rounding, to E4M3, picks the code the exact quotient would.
+__device__ __forceinline__ float e4m3_prescale(float h, float amax, float pre) {
+  return __fdiv_rn(__fmul_rn(__fmul_rn(h, pre), 448.f), __fmul_rn(amax, pre));
+}
+// pre: 2^-64 for rows with a huge amax, so that h * 448 cannot overflow (powers of two: exact)
+__device__ __forceinline__ float e4m3_pre(float amax) { return amax > 0x1p100f ? 0x1p-64f : 1.f; }
 __global__ void __launch_bounds__(256) quantize_rows_kernel(CallParams cp, Workspace ws,
                                                             const __nv_bfloat16* __restrict__ H) {
   __shared__ float s_p[8];
@@ -233,11 +241,12 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(CallParams cp, Works
   }
   __syncthreads();
   amax = s_amax;
-  const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+  const float pre = e4m3_pre(amax);
+  const float den = amax > 0.f ? amax : 1.f;   // an all-zero row quantises to zeros
   uint8_t* out = ws.h8 + (size_t)row * cp.d;
   for (int k = 2 * threadIdx.x; k < cp.d; k += 2 * blockDim.x) {
-    const float a = __fmul_rn(__bfloat162float(h[k]), inv);
-    const float b = k + 1 < cp.d ? __fmul_rn(__bfloat162float(h[k + 1]), inv) : 0.f;
+    const float a = e4m3_prescale(__bfloat162float(h[k]), den, pre);
+    const float b = k + 1 < cp.d ? e4m3_prescale(__bfloat162float(h[k + 1]), den, pre) : 0.f;
     unsigned short pair;   // upper byte = code of the first operand, lower byte = code of the second
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair) : "f"(b), "f"(a));
     out[k] = (uint8_t)(pair & 0xFF);
@@ -247,7 +256,7 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(CallParams cp, Works
 
 // The same quantisation for d % 8 == 0: the row is read once, eight bf16 per 16-byte load, kept
 // in registers across the amax reduction, and written as eight codes per store. kVec = loads
-// per thread (blockDim.x * kVec * 8 >= d). Same float32 operations per element as above.
+// per thread (blockDim.x * kVec * 8 >= d). Same operations per element as above.
 template <int kVec>
 __global__ void __launch_bounds__(1024) quantize_rows_vec_kernel(CallParams cp, Workspace ws,
                                                                  const __nv_bfloat16* __restrict__ H) {
@@ -283,7 +292,8 @@ __global__ void __launch_bounds__(1024) quantize_rows_vec_kernel(CallParams cp, 
   }
   __syncthreads();
   amax = s_amax;
-  const float inv = amax > 0.f ? __fdiv_rn(448.f, amax) : 0.f;
+  const float pre = e4m3_pre(amax);
+  const float den = amax > 0.f ? amax : 1.f;   // an all-zero row quantises to zeros
   uint2* out = reinterpret_cast<uint2*>(ws.h8 + (size_t)row * cp.d);
 #pragma unroll
   for (int u = 0; u < kVec; ++u) {
@@ -293,8 +303,8 @@ __global__ void __launch_bounds__(1024) quantize_rows_vec_kernel(CallParams cp, 
     uint32_t pair[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const float a = __fmul_rn(__uint_as_float(w[q] << 16), inv);           // element 2q
-      const float b = __fmul_rn(__uint_as_float(w[q] & 0xFFFF0000u), inv);   // element 2q + 1
+      const float a = e4m3_prescale(__uint_as_float(w[q] << 16), den, pre);           // element 2q
+      const float b = e4m3_prescale(__uint_as_float(w[q] & 0xFFFF0000u), den, pre);   // element 2q + 1
       unsigned short p;   // upper byte = code of the first operand, lower byte = code of the second
       asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(p) : "f"(b), "f"(a));
       pair[q] = p;
@@ -538,7 +548,7 @@ static void simt_logits(const CallParams& cp, const Workspace& ws, const void* W
 }
 
 int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const float* w_scale, const void* w_judge,
-             const void* H, int dtype, float* logits_debug, cudaStream_t st) {
+             const void* H, int dtype, cudaStream_t st) {
   const int np = (cp.V + kVocabTile - 1) / kVocabTile;
   auto logits = [&](int mode, float* dbg) {
     if (dtype == JD_DTYPE_FP8_E4M3)   // E4M3 weights against the E4M3 rows the caller quantised into ws.h8
@@ -548,7 +558,7 @@ int run_simt(const CallParams& cp, const Workspace& ws, const void* W, const flo
   };
   const int nq = launch_q_stats(cp, ws, st);
   launch_judge(cp, ws, H, w_judge, dtype == JD_DTYPE_F32 ? JD_DTYPE_F32 : JD_DTYPE_BF16, st);
-  logits(0, logits_debug);
+  logits(0, cp.logits_debug);
   launch_fold(cp, ws, np, nq, st);
   if (cp.rule == JD_RULE_TOPK) {   // ranks and argmax need the folded maxima; the decision writes the token
     logits(2, nullptr);

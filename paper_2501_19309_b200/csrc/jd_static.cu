@@ -13,6 +13,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <mutex>
 
 #include "jd_kernels.h"
 
@@ -61,6 +62,9 @@ bool encode_bf16_rows(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+std::mutex g_setup_mutex;   // first calls from several host threads set a device up once
 
 }  // namespace
 
@@ -78,6 +82,10 @@ extern "C" jd_status_t jd_verify_static(int32_t d, int32_t V, const void* W, con
   if (a->rule != JD_RULE_SAMPLING) return JD_ERR_UNSUPPORTED;   // the fixed scratch has no rank counters
   if (a->norm != JD_NORM_NONE) return JD_ERR_UNSUPPORTED;       // nor row normalisation factors
   if (!aligned16(W) || !aligned16(w_judge) || !aligned16(a->H)) return JD_ERR_INVALID_ARG;
+  if (!aligned4(a->draft_tokens) || !aligned4(a->draft_logits) || !aligned4(a->accept_len) || !aligned4(a->next_token) ||
+      !aligned4(a->judge_scores) || !aligned4(a->p_draft) || !aligned4(a->q_draft) || !aligned4(a->row_max) ||
+      !aligned4(a->row_lse) || !aligned4(device_status))
+    return JD_ERR_INVALID_ARG;
   // the fixed scratch holds at most 96 rows: larger blocks are refused, never truncated
   if ((int64_t)a->B * (a->M + 1) > kStaticMaxRows) return JD_ERR_UNSUPPORTED;
   const int R = a->B * (a->M + 1);
@@ -85,22 +93,25 @@ extern "C" jd_status_t jd_verify_static(int32_t d, int32_t V, const void* W, con
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return JD_ERR_CUDA;
   if (dev < 0 || dev >= kMaxDevices) return JD_ERR_UNSUPPORTED;
+  std::unique_lock<std::mutex> setup_lock(g_setup_mutex);
   if (!g_scratch_ptr[dev]) {
-    // one-time set-up on this device (it is the current one): architecture, SM count, and the
-    // device address of the scratch array
+    // one-time set-up on this device (it is the current one): architecture, SM count, the device
+    // address of the scratch array, and the kernels themselves (their shared-memory limit is raised
+    // here, which also loads every instantiation, so that no later call has to load code)
     int major = 0, sms = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return JD_ERR_CUDA;
     if (major != 10) return JD_ERR_ARCH;
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p || !fused_configure()) {
       cudaGetLastError();
       return JD_ERR_CUDA;
     }
     g_num_sms[dev] = sms;
     g_scratch_ptr[dev] = p;
   }
+  setup_lock.unlock();
 
   FusedPlan plan;
   if (!fused_supported(JD_DTYPE_BF16, R, d, V, g_num_sms[dev], &plan)) return JD_ERR_UNSUPPORTED;
@@ -140,6 +151,8 @@ extern "C" jd_status_t jd_verify_static(int32_t d, int32_t V, const void* W, con
   cp.judge_scores = a->judge_scores; cp.p_draft = a->p_draft;
   cp.q_draft = a->q_draft; cp.masks = a->masks;
   cp.row_max_out = a->row_max; cp.row_lse_out = a->row_lse;
+  cp.logits_debug = nullptr;
+  cp.dl_vec4 = (V % 4 == 0 && aligned16(a->draft_logits)) ? 1 : 0;   // else the kernel's 4-byte loads
 
   CUtensorMap tm_w, tm_h;
   if (!encode_bf16_rows(&tm_w, W, (uint64_t)V, (uint64_t)d, 128) ||

@@ -33,7 +33,8 @@ VARIANTS = {"auto": JD_VARIANT_AUTO, "simt": JD_VARIANT_SIMT, "fused": JD_VARIAN
 
 EXPORTS = ["jd_version", "jd_status_string", "jd_workspace_bytes", "jd_create", "jd_destroy", "jd_set_head",
            "jd_verify", "jd_verify_host", "jd_last_device_status", "jd_last_launch_info", "jd_philox_uniforms",
-           "jd_verify_static", "jd_set_head_fp8", "jd_selftest_timeout", "jd_stream_read_probe"]
+           "jd_verify_static", "jd_set_head_fp8", "jd_selftest_timeout", "jd_stream_read_probe",
+           "jd_quantize_rows_e4m3", "jd_check_workspace_guards"]
 
 
 class jd_config_t(C.Structure):
@@ -88,6 +89,8 @@ def load():
     lib.jd_stream_read_probe.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
     lib.jd_verify_static.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_float,
                                      C.POINTER(jd_verify_args_t), C.c_void_p, C.c_void_p]
+    lib.jd_quantize_rows_e4m3.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.jd_check_workspace_guards.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
     for name in EXPORTS:
         if name not in ("jd_version", "jd_status_string", "jd_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -166,6 +169,21 @@ def jd_stream_read_probe(data_ptr: int, nbytes: int, out_ptr: int, stream_ptr: i
     """Reads nbytes at data_ptr once and XORs every 32-bit word into the word at out_ptr; see jd.h."""
     return load().jd_stream_read_probe(C.c_void_p(data_ptr), C.c_size_t(nbytes), C.c_void_p(out_ptr),
                                        C.c_void_p(stream_ptr))
+
+
+def jd_quantize_rows_e4m3(H_ptr: int, rows: int, d: int, codes_ptr: int, scale_ptr: int, stream_ptr: int = 0) -> int:
+    """The library's per-row E4M3 quantiser on its own (test helper); see jd.h."""
+    return load().jd_quantize_rows_e4m3(C.c_void_p(H_ptr), C.c_int32(rows), C.c_int32(d), C.c_void_p(codes_ptr),
+                                        C.c_void_p(scale_ptr), C.c_void_p(stream_ptr))
+
+
+def jd_check_workspace_guards(h) -> int:
+    """Number of damaged guard blocks between the handle's workspace regions (0 = intact)."""
+    out = C.c_int32(-1)
+    st = load().jd_check_workspace_guards(h, C.byref(out))
+    if st != JD_OK:
+        raise JdError(st, "jd_check_workspace_guards")
+    return out.value
 
 
 def jd_verify_static(d: int, V: int, W_ptr: int, w_judge_ptr: int, b_judge: float, args: jd_verify_args_t,
@@ -298,3 +316,6 @@ class Verifier:
 
     def launch_info(self):
         return jd_last_launch_info(self.h)
+
+    def damaged_guards(self) -> int:
+        return jd_check_workspace_guards(self.h)

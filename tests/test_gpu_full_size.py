@@ -1,6 +1,7 @@
 """Parity at the published workload sizes, in the launch configuration the benchmark times
-(variant chosen automatically).  The CPU checker recomputes whole sequences; where a workload
-has several sequences a sample of them is checked."""
+(variant chosen automatically): every listed configuration, mode, seed and threshold against the
+CPU checker, which recomputes whole sequences.  Every case adds its counts (margin exemptions,
+exactly equal next tokens, largest deviations) to the session's parity table."""
 import numpy as np
 import pytest
 
@@ -9,9 +10,13 @@ from paper_2501_19309_b200 import inputs as I
 
 pytestmark = pytest.mark.gpu
 
+ALL_MODES = ("standard", "judge", "judge_or_standard")
 
-def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None, rule="sampling", top_k=1, fp8=False):
-    """cases: list of (mode, tau or None)."""
+
+def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None, rule="sampling", top_k=1, fp8=False,
+              check_logits=False, label=None):
+    """cases: list of (mode, tau or None). Returns (report, inputs, outputs of the last case)."""
+    import torch
     from paper_2501_19309_b200 import jd
     wl = I.CONFIGS[cfg]
     if fp8:
@@ -20,54 +25,54 @@ def full_case(cfg, data_seed, cases, sequences=None, expect_variant=None, rule="
     dev = T.upload(inp)
     ver = T.make_verifier(inp, dev)
     rep = T.Report()
+    got = None
     for mode, tau in cases:
         tau = inp.tau if tau is None else tau
-        out = ver.verify(dev["H"], dev["x"], dev["dl"], tau, inp.seed, mode, rule=rule, top_k=top_k)
+        out = ver.alloc_outputs(wl.B, wl.M, debug_logits=check_logits)
+        ver.verify(dev["H"], dev["x"], dev["dl"], tau, inp.seed, mode, rule=rule, top_k=top_k, out=out)
         assert ver.device_status() == jd.JD_OK
         if expect_variant:
             assert ver.launch_info()[0] == jd.VARIANTS[expect_variant]
         got = T.to_numpy(out)
-        ref = T.run_oracle(inp, mode, tau=tau, sequences=sequences, rule=rule, top_k=top_k)
+        ref = T.run_oracle(inp, mode, tau=tau, sequences=sequences, rule=rule, top_k=top_k, keep_logits=check_logits)
         T.compare(got, ref, mode, wl.M, rep, rule=rule)
+        if check_logits:
+            T.compare_logits(got["logits_debug"], ref, rep)
+    assert ver.damaged_guards() == 0
+    if fp8:
+        assert T.fp8_row_code_mismatches(inp, dev) == 0
     ver.close()
     del dev
-    import torch
     torch.cuda.empty_cache()
-    print("\n%s: %s" % (wl.name, rep))
-    return rep, inp
+    T.record(label or (wl.name + ("" if rule == "sampling" else "-top%d" % top_k)), rep)
+    return rep, inp, got
 
 
-@pytest.mark.parametrize("data_seed", [0, 1])
-def test_cfg1_8b_head(data_seed):
+@pytest.mark.parametrize("data_seed", range(10))
+def test_cfg1_8b_head_every_seed_and_threshold(data_seed):
+    """Seeds 0..9 (data seed = verify seed), the threshold sweep on each; the two single-test modes on
+    seed 0, together with the element-wise logits of the tensor-core kernel."""
     cases = [("judge_or_standard", 0.3), ("judge_or_standard", 0.5), ("judge_or_standard", 0.7)]
     if data_seed == 0:
         cases += [("standard", None), ("judge", None)]
-    full_case(1, data_seed, cases, expect_variant="fused")
+    rep, _, _ = full_case(1, data_seed, cases, expect_variant="fused", check_logits=(data_seed == 0))
+    assert rep.sequences == len(cases)
+    if data_seed == 0:
+        assert 0 < rep.max_rel_logit <= T.REL_TOL
 
 
-def test_cfg2_70b_head_sampled_sequences():
-    rep, _ = full_case(2, 0, [("judge_or_standard", None)], sequences=[0, 3], expect_variant="fused")
-    assert rep.sequences == 2
+def test_cfg2_70b_head_every_sequence():
+    rep, _, _ = full_case(2, 0, [("judge_or_standard", None)], expect_variant="fused")
+    assert rep.sequences == 4
 
 
-def test_cfg3_405b_head_forced_rejection():
-    from paper_2501_19309_b200 import jd
+def test_cfg3_405b_head_all_modes_forced_rejection():
     wl = I.CONFIGS[3]
-    inp = I.make_inputs(wl, 0)
-    dev = T.upload(inp)
-    ver = T.make_verifier(inp, dev)
-    rep = T.Report()
-    for mode in ("standard", "judge", "judge_or_standard"):
-        out = ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau, inp.seed, mode)
-        assert ver.device_status() == jd.JD_OK and ver.launch_info()[0] == jd.JD_VARIANT_FUSED
-        got = T.to_numpy(out)
+    for mode in ALL_MODES:
+        rep, inp, got = full_case(3, 0, [(mode, None)], expect_variant="fused")
+        assert rep.sequences == 1
         assert got["accept_len"][0] <= wl.forced_reject_at           # rejection forced at slot 12
         assert got["masks"][0, wl.forced_reject_at] == 0
-        if mode == "judge_or_standard":                              # one full checker pass (the slow part)
-            ref = T.run_oracle(inp, mode)
-            T.compare(got, ref, mode, wl.M, rep)
-    ver.close()
-    print("\ncfg3:", rep)
 
 
 def test_cfg3_masks_independent_of_mode():
@@ -75,8 +80,7 @@ def test_cfg3_masks_independent_of_mode():
     inp = I.make_inputs(wl, 0)
     dev = T.upload(inp)
     ver = T.make_verifier(inp, dev)
-    masks = [T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau, 0, m))["masks"]
-             for m in ("standard", "judge", "judge_or_standard")]
+    masks = [T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau, 0, m))["masks"] for m in ALL_MODES]
     assert np.array_equal(masks[0], masks[1]) and np.array_equal(masks[0], masks[2])
     for mode in ("standard", "judge"):
         got = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau, 0, mode))
@@ -84,9 +88,30 @@ def test_cfg3_masks_independent_of_mode():
     ver.close()
 
 
-def test_cfg4_batched_sampled_sequences():
-    rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[0, 37, 63], expect_variant="batched")
-    assert rep.sequences == 3
+def test_cfg4_batched_every_sequence_against_checker_and_cuda_core_variant():
+    """Seed 0: all 64 sequences against the CPU checker, and against the CUDA-core variant on the
+    device at full d and V."""
+    import torch
+    rep, inp, got = full_case(4, 0, [("judge_or_standard", None)], expect_variant="batched")
+    assert rep.sequences == 64
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    ref = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], inp.tau, inp.seed, "judge_or_standard", variant="simt"))
+    assert np.array_equal(got["accept_len"], ref["accept_len"])
+    assert np.array_equal(got["masks"], ref["masks"])
+    assert np.allclose(got["row_lse"], ref["row_lse"], rtol=0, atol=2e-4)
+    assert np.allclose(got["p_draft"], ref["p_draft"], rtol=2e-4)
+    assert np.allclose(got["judge_scores"], ref["judge_scores"], rtol=0, atol=T.JUDGE_ABS_TOL)
+    ver.close()
+    del dev
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("data_seed", [1, 2, 3, 4])
+def test_cfg4_remaining_seeds_eight_sequences_each(data_seed):
+    seqs = [(7 * data_seed + 8 * i) % 64 for i in range(8)]
+    rep, _, _ = full_case(4, data_seed, [("judge_or_standard", None)], sequences=seqs, expect_variant="batched")
+    assert rep.sequences == 8
 
 
 def test_cfg1_greedy_and_top5_rules():
@@ -95,30 +120,17 @@ def test_cfg1_greedy_and_top5_rules():
 
 
 def test_cfg4_greedy_rule_sampled_sequences():
-    rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[5, 60], expect_variant="batched",
-                       rule="topk", top_k=1)
-    assert rep.sequences == 2
+    rep, _, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[5, 21, 40, 60], expect_variant="batched",
+                          rule="topk", top_k=1)
+    assert rep.sequences == 4
 
 
 def test_cfg3_fp8_head_full_size():
-    rep, _ = full_case(3, 0, [("judge_or_standard", None)], expect_variant="fused", fp8=True)
+    rep, _, _ = full_case(3, 0, [("judge_or_standard", None)], expect_variant="fused", fp8=True)
     assert rep.sequences == 1
 
 
 def test_cfg4_fp8_head_sampled_sequences():
-    rep, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=[0, 63], expect_variant="batched", fp8=True)
-    assert rep.sequences == 2
-
-
-@pytest.mark.parametrize("data_seed", [2, 3, 4, 5, 6, 7, 8, 9])
-def test_cfg1_remaining_seeds(data_seed):
-    """Seeds 0 and 1 run the whole threshold sweep above; the other eight of the workload's ten seeds
-    (data seed = verify seed) run the paper's mode at tau = 0.5."""
-    full_case(1, data_seed, [("judge_or_standard", 0.5)], expect_variant="fused")
-
-
-@pytest.mark.parametrize("data_seed", [1, 2, 3, 4])
-def test_cfg4_remaining_seeds_one_sequence_each(data_seed):
-    rep, _ = full_case(4, data_seed, [("judge_or_standard", None)], sequences=[(17 * data_seed) % 64],
-                       expect_variant="batched")
-    assert rep.sequences == 1
+    rep, _, _ = full_case(4, 0, [("judge_or_standard", None)], sequences=list(range(0, 64, 8)),
+                          expect_variant="batched", fp8=True)
+    assert rep.sequences == 8

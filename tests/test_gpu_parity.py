@@ -13,7 +13,7 @@ MODES = ("standard", "judge", "judge_or_standard")
 
 
 def run_case(wl, data_seed, modes=MODES, variant="auto", seeds=None, tau=None, check_logits=False,
-             sequences=None, expect_variant=None, rule="sampling", top_k=1, rms_eps=None):
+             sequences=None, expect_variant=None, rule="sampling", top_k=1, rms_eps=None, record_as=None):
     from paper_2501_19309_b200 import jd
     inp = I.make_inputs(wl, data_seed)
     dev = T.upload(inp)
@@ -33,7 +33,12 @@ def run_case(wl, data_seed, modes=MODES, variant="auto", seeds=None, tau=None, c
             T.compare(got, ref, mode, wl.M, rep, rule=rule)
             if check_logits:
                 T.compare_logits(got["logits_debug"], ref, rep)
+    assert ver.damaged_guards() == 0          # no kernel wrote past the end of a workspace region
+    if wl.dtype == "fp8":
+        assert T.fp8_row_code_mismatches(inp, dev) == 0
     ver.close()
+    if record_as:
+        T.record(record_as, rep, bound=False)
     return rep
 
 
@@ -166,12 +171,44 @@ def test_argument_validation_returns_codes():
     a3, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, out=out)
     a3.H = dev["H"].data_ptr() + 2                           # misaligned
     assert jd.jd_verify(ver.h, a3) == jd.JD_ERR_INVALID_ARG
+    for field in ("draft_logits", "draft_tokens", "accept_len", "judge_scores", "q_draft", "row_lse"):
+        a5, _ = ver.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, out=out)
+        setattr(a5, field, getattr(a5, field) + 2)           # a float / int32 array off its 4-byte boundary
+        assert jd.jd_verify(ver.h, a5) == jd.JD_ERR_INVALID_ARG, field
     v2 = jd.Verifier(2, 3, wl.d, wl.V, "bf16")
     a4, _ = v2.make_args(dev["H"], dev["x"], dev["dl"], 0.5, 0, out=out)
     assert jd.jd_verify(v2.h, a4) == jd.JD_ERR_INVALID_ARG   # no head registered yet
     v2.close()
     with pytest.raises(jd.JdError):
         jd.jd_create(jd.jd_config_t(1, 1, 64, 600, 5, 0))
+    ver.close()
+
+
+@pytest.mark.parametrize("variant,B,M,d,V", [("fused", 2, 5, 128, 40000), ("simt", 2, 5, 96, 4000),
+                                             ("batched", 12, 9, 128, 20000)])
+def test_draft_logits_view_that_is_only_4_byte_aligned(variant, B, M, d, V):
+    """A slice of a larger buffer: the draft logits start one float past a 16-byte boundary although
+    V % 4 == 0. The kernels must take their 4-byte loads (never a misaligned 16-byte one) and give
+    the same results as for an aligned copy."""
+    import torch
+    wl = I.CONFIGS[2].scaled("dlview-" + variant, B=B, M=M, d=d, V=V)
+    inp = I.make_inputs(wl, 21)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    big = torch.empty(dev["dl"].numel() + 8, dtype=torch.float32, device="cuda")
+    assert big.data_ptr() % 16 == 0
+    view = big[1:1 + dev["dl"].numel()].view(B, M, V)
+    view.copy_(dev["dl"])
+    assert view.data_ptr() % 16 == 4 and view.is_contiguous()
+    for seed in (0, 1):
+        want = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, seed, "judge_or_standard", variant=variant))
+        got = T.to_numpy(ver.verify(dev["H"], dev["x"], view, 0.5, seed, "judge_or_standard", variant=variant))
+        from paper_2501_19309_b200 import jd
+        assert ver.device_status() == jd.JD_OK
+        T.compare(got, T.run_oracle(inp, "judge_or_standard", seed=seed), "judge_or_standard", M)
+        for k in ("accept_len", "masks", "next_token"):
+            assert np.array_equal(want[k], got[k]), k
+        assert np.allclose(want["q_draft"], got["q_draft"], rtol=1e-5)
     ver.close()
 
 
@@ -209,8 +246,9 @@ FUSED_SHAPES = [
 @pytest.mark.parametrize("B,M,d,V", FUSED_SHAPES)
 def test_fused_variant_parity(B, M, d, V):
     wl = I.CONFIGS[2].scaled("fused-%d-%d-%d-%d" % (B, M, d, V), B=B, M=M, d=d, V=V)
-    rep = run_case(wl, 3, variant="fused", seeds=[0, 1], expect_variant="fused")
-    assert rep.sequences == 6 * B
+    rep = run_case(wl, 3, variant="fused", seeds=[0, 1], expect_variant="fused", check_logits=True,
+                   record_as="small-shapes-fused")
+    assert rep.sequences == 6 * B and 0 < rep.max_rel_logit <= T.REL_TOL
 
 
 def test_fused_matches_simt_variant_on_device():
@@ -259,8 +297,8 @@ def test_batched_variant_parity(B, M, d, V):
     wl = I.CONFIGS[4].scaled("batched-%d-%d-%d-%d" % (B, M, d, V), B=B, M=M, d=d, V=V)
     seqs = None if B <= 8 else sorted({0, 1, B // 2, B - 1})
     rep = run_case(wl, 5, variant="batched", modes=("judge_or_standard", "standard"), seeds=[0, 1],
-                   sequences=seqs, expect_variant="batched")
-    assert rep.sequences == 4 * (B if seqs is None else len(seqs))
+                   sequences=seqs, expect_variant="batched", check_logits=True, record_as="small-shapes-batched")
+    assert rep.sequences == 4 * (B if seqs is None else len(seqs)) and 0 < rep.max_rel_logit <= T.REL_TOL
 
 
 @pytest.mark.parametrize("B,M", [(48, 7), (150, 3)])
@@ -343,7 +381,7 @@ def test_rms_normalised_head_parity(variant, B, M, d, V, dtype):
                              alpha_range=(2.0, 9.0))           # rows of clearly different norms
     seqs = None if B <= 8 else [0, B // 2, B - 1]
     rep = run_case(wl, 11, variant=variant, modes=("judge_or_standard", "standard"), seeds=[0, 1],
-                   sequences=seqs, expect_variant=variant, rms_eps=1e-5, check_logits=(variant == "simt"))
+                   sequences=seqs, expect_variant=variant, rms_eps=1e-5, check_logits=True)
     assert rep.sequences == 4 * (B if seqs is None else len(seqs))
     if variant == "fused":
         rep = run_case(wl, 11, variant=variant, modes=("standard",), seeds=[0], rule="greedy", rms_eps=1e-5)
@@ -383,8 +421,8 @@ FP8_CASES = [
 def test_fp8_head_parity(variant, B, M, d, V):
     wl = I.CONFIGS[2].scaled("fp8-%s-%d-%d-%d-%d" % (variant, B, M, d, V), B=B, M=M, d=d, V=V, dtype="fp8")
     rep = run_case(wl, 13, variant=variant, modes=("judge_or_standard", "standard"), seeds=[0, 1],
-                   expect_variant=variant, check_logits=(variant == "simt"))
-    assert rep.sequences == 4 * B
+                   expect_variant=variant, check_logits=True, record_as="small-shapes-fp8-" + variant)
+    assert rep.sequences == 4 * B and 0 < rep.max_rel_logit <= T.REL_TOL
     if variant != "simt":
         run_case(wl, 13, variant=variant, modes=("standard",), seeds=[0], rule="greedy", rms_eps=1e-5)
         run_case(wl, 13, variant=variant, modes=("judge_or_standard",), seeds=[0], rule="topk", top_k=7)

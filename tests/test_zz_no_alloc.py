@@ -6,7 +6,9 @@ not pay the synchronisation an allocation implies.  The entry point keeps the fu
 scratch in a fixed array inside the library, so the test checks two things through the C ABI:
 that it gives exactly what jd_verify (fused variant, handle-owned scratch) gives, and that a
 second call right after the first, on a different and smaller block, is not disturbed by what
-the first call left in the shared array.  Floating-point outputs are compared with the tolerance
+the first call left in the shared array.  Both calls are also compared with the CPU checker, so
+the test does not rest on the handle path alone, and the device's free memory is read before
+and after them: it must not move.  Floating-point outputs are compared with the tolerance
 the other GPU tests use (relative 2e-3; judge scores 2e-5), integer outputs must be equal.
 This file sorts last on purpose: a run that stops at the first failure has then already run
 every other test.
@@ -46,17 +48,38 @@ def test_static_entry_point_matches_handle_path_on_two_calls_in_a_row():
 
     status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream().cuda_stream
+    # output buffers first, then one warm-up call (the first call on a device looks up the scratch
+    # address and loads the kernels); from here on the free memory of the device must stay put
+    prepared = [ver.make_args(dev["H"], dev["x"], dev["dl"], inp.tau, seed, "judge_or_standard")
+                for wl, inp, dev, ver, seed, want in calls]
+    wl, inp, dev, ver, seed, _ = calls[1]
+    assert jd.jd_verify_static(wl.d, wl.V, dev["W"].data_ptr(), dev["w"].data_ptr(), inp.b_judge, prepared[1][0],
+                               status.data_ptr(), stream) == jd.JD_OK
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     outs = []
-    for wl, inp, dev, ver, seed, want in calls:                # back to back, no sync in between
-        args, out = ver.make_args(dev["H"], dev["x"], dev["dl"], inp.tau, seed, "judge_or_standard")
+    for (wl, inp, dev, ver, seed, want), (args, out) in zip(calls, prepared):   # back to back, no sync in between
         st = jd.jd_verify_static(wl.d, wl.V, dev["W"].data_ptr(), dev["w"].data_ptr(), inp.b_judge, args,
                                  status.data_ptr(), stream)
         assert st == jd.JD_OK, jd.jd_status_string(st)
         outs.append(out)
     torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before         # nothing was allocated on the device
     assert int(status.item()) == jd.JD_OK
     for (wl, inp, dev, ver, seed, want), out in zip(calls, outs):
-        _same(T.to_numpy(out), want)
+        got = T.to_numpy(out)
+        _same(got, want)
+        T.compare(got, T.run_oracle(inp, "judge_or_standard", seed=seed), "judge_or_standard", wl.M)
+
+    # a draft token outside the vocabulary is clamped and reported in the caller's status word
+    wl, inp, dev, ver, seed, _ = calls[1]
+    x_bad = dev["x"].clone()
+    x_bad[0, 2] = wl.V + 9
+    args, _ = ver.make_args(dev["H"], x_bad, dev["dl"], inp.tau, seed)
+    assert jd.jd_verify_static(wl.d, wl.V, dev["W"].data_ptr(), dev["w"].data_ptr(), inp.b_judge, args,
+                               status.data_ptr(), stream) == jd.JD_OK
+    torch.cuda.synchronize()
+    assert int(status.item()) == jd.JD_ERR_BAD_TOKEN
 
     # sizes beyond the fixed scratch are refused with a clear status, nothing is launched
     wl, inp, dev, ver, seed, _ = calls[0]

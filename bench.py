@@ -40,6 +40,7 @@ if ROOT not in sys.path:
 
 from paper_2501_19309_b200 import inputs as I  # noqa: E402
 
+T_START = time.perf_counter()
 METRIC = "verified_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -298,9 +299,17 @@ def run_reference(args, wl) -> None:
     print(json.dumps(line), flush=True)
 
 
+def log(msg: str) -> None:
+    """Progress on stderr (the JSON line is the only thing on stdout)."""
+    sys.stderr.write("[bench %7.1f s] %s\n" % (time.perf_counter() - T_START, msg))
+    sys.stderr.flush()
+
+
 def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     """Times K device-resident calls and K_e2e host-buffer calls of one workload on this rank."""
+    log("%s: drawing inputs" % wl.name)
     inp = I.make_inputs(wl, data_seed)
+    log("%s: inputs drawn" % wl.name)
     fp8 = wl.dtype == "fp8"
     W = torch.from_numpy(inp.W).to(device) if fp8 else torch.from_numpy(inp.W).view(torch.bfloat16).to(device)
     w_scale = torch.from_numpy(inp.w_scale).to(device) if fp8 else None
@@ -419,6 +428,7 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     h2d = hH.numel() * 2 + hx.numel() * 4 + hdl.numel() * 4
     d2h = sum(hout[k].numel() * hout[k].element_size() for k in hout)
     ver.close()
+    log("%s: measured" % wl.name)
     res = dict(total_ms=total_ms, median_ms=statistics.median(per), min_ms=min(per), mean_ms=total_ms / K,
                variant=variant, launches=launches, clocks=clocks, e2e_s=e2e_s, e2e_steps=Ke, h2d=h2d, d2h=d2h,
                mean_accept=float(accepted.mean()), emitted_per_call=float((accepted + 1).sum(axis=1).mean()),
@@ -496,8 +506,8 @@ def main() -> None:
             small.e2e_steps = 10
             r = measure_workload(owl, small, torch, jd, device, data_seed=0, sample_clocks=True)
             oparity = None
-            if not args.no_cpu_baseline:      # a few seconds of the checker on the first sequences
-                oparity = parity_of(owl, r["out0"], time_oracle(r["inp"], 1, budget_s=5.0)["first"])
+            if not args.no_cpu_baseline:      # the checker on the first sequence of this workload
+                oparity = parity_of(owl, r["out0"], oracle_step(r["inp"], 0, [0]))
             e2e_note = None
             if owl.B * owl.M * owl.V * 4 > 100e6:
                 e2e_note = ("%.0f MB of fp32 draft logits cross PCIe per host-buffer call" % (owl.B * owl.M * owl.V * 4 / 1e6))
@@ -518,6 +528,7 @@ def main() -> None:
 
     if rank == 0:
         cpu, parity = None, None
+        log("workloads done; CPU baseline")
         if not args.no_cpu_baseline:
             c = time_oracle(res["inp"], 1)
             cpu = {k: c[k] for k in ("value", "unit", "cores", "kind", "sample")}

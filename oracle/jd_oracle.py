@@ -139,15 +139,21 @@ def _to_f64(a: np.ndarray) -> np.ndarray:
 # --------------------------------------------------------------------------
 # FP8 E4M3 ("fn": finite, no infinities; 0x7F / 0xFF are NaN), from the format's definition
 # --------------------------------------------------------------------------
+def _e4m3_value(c: int) -> float:
+    """Value of one E4M3 code: (-1)^s 2^(e-7) (1 + m/8); e = 0: (-1)^s 2^-6 m/8; 0x7F / 0xFF: NaN."""
+    s, e, m = c >> 7, (c >> 3) & 0xF, c & 0x7
+    if e == 0xF and m == 0x7:
+        return float("nan")
+    mag = (m / 8.0) * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return -mag if s else mag
+
+
+_E4M3_TABLE = np.array([_e4m3_value(c) for c in range(256)], dtype=np.float64)
+
+
 def e4m3_decode(codes: np.ndarray) -> np.ndarray:
-    """float64 values of E4M3 codes (uint8): (-1)^s 2^(e-7) (1 + m/8), e = 0: (-1)^s 2^-6 m/8."""
-    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
-    sgn = np.where(c & 0x80, -1.0, 1.0)
-    e = (c >> 3) & 0xF
-    m = (c & 0x7).astype(np.float64)
-    val = np.where(e == 0, np.ldexp(m / 8.0, -6), np.ldexp(1.0 + m / 8.0, e - 7))
-    val = np.where((c & 0x7F) == 0x7F, np.nan, val)
-    return sgn * val
+    """float64 values of E4M3 codes (uint8): the 256 values of the format, looked up by code."""
+    return _E4M3_TABLE[np.asarray(codes, dtype=np.uint8)]
 
 
 def e4m3_round(x: np.ndarray) -> np.ndarray:

@@ -58,7 +58,6 @@ struct FusedParams {
   int tile_stride;  // TMEM columns between consecutive tiles (>= rows, multiple of 8, <= N_PAD)
   int R;            // rows of the H matrix given to the MMA: B * (M + 1), or B in sample-only mode
   int fp8;          // 1: W and H tiles hold FP8 E4M3 codes (128 per 128-byte row), kind::f8f6f4 MMAs
-  int sample_only;  // 1: H holds one already selected row per sequence; only the token draw runs
   int late_tiles;   // > 0: a CTA whose tiles all fit in TMEM finishes all but its last `late_tiles` tiles first
                     // (own sweep over d), so that their row statistics are taken while the rest still streams
   // Host-buffer calls: the draft logits may still be on their way to the device when the kernel
@@ -183,7 +182,13 @@ __device__ __noinline__ void dump_logits(float* __restrict__ out, int T, int t0,
 
 // kFp8 is a template parameter, not a runtime flag: a kernel whose MMA loop can reach both
 // tcgen05.mma kinds ran its bf16 main loop 40 % slower.
-template <int N_PAD, bool kFp8>
+// kKind selects what the epilogue contains, so that each instantiation carries only its own code:
+//   kFullSampling  the whole verification step with the stochastic test of Eq. 4 and the token draw
+//   kFullTopK      the whole step with the deterministic top-K / greedy rule (rank counts, argmax)
+//   kSampleOnly    H holds one already selected row per sequence; only the token draw runs
+enum : int { kFullSampling = 0, kFullTopK = 1, kSampleOnlyKind = 2 };
+
+template <int N_PAD, bool kFp8, int kKind>
 __global__ void __launch_bounds__(kThreads, 1)
 fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, CallParams cp,
                     Workspace ws, const __nv_bfloat16* __restrict__ H, const __nv_bfloat16* __restrict__ wj,
@@ -200,6 +205,8 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, G = gridDim.x;
   volatile int* abort_flag = &ms.abort_flag;
+  constexpr bool kSampleOnly = (kKind == kSampleOnlyKind);
+  constexpr bool kTopK = (kKind == kFullTopK);
 
   // vocabulary tiles of this CTA
   const int base = fp.num_tiles / G, rem = fp.num_tiles % G;
@@ -224,7 +231,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   }
   if (tid < N_PAD) {
     int x = -1;
-    if (tid < R && !fp.sample_only) {
+    if (tid < R && !kSampleOnly) {
       const int b = tid / (M + 1), j = tid % (M + 1);
       if (j < M) {
         x = cp.draft_tokens[b * M + j];
@@ -233,8 +240,8 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     ms.x_row[tid] = x;
     float f = 1.f;   // normalisation factor of the row held in TMEM column tid
-    if (cp.norm == JD_NORM_RMS && tid < R) f = ws.row_scale[fp.sample_only ? ws.sel_row[tid] : tid];
-    if (fp.fp8 && tid < R) f *= ws.h_scale[fp.sample_only ? ws.sel_row[tid] : tid];
+    if (cp.norm == JD_NORM_RMS && tid < R) f = ws.row_scale[kSampleOnly ? ws.sel_row[tid] : tid];
+    if (fp.fp8 && tid < R) f *= ws.h_scale[kSampleOnly ? ws.sel_row[tid] : tid];
     ms.scale[tid] = f;
   }
   if (tid < kVocabTile) {   // per-vocabulary-row scales of an FP8 head, one per tile of this CTA; 1 otherwise
@@ -390,7 +397,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     const int v_lo = t0 * kVocabTile, v_hi = min(V, (t0 + T) * kVocabTile);
     const bool vec4 = cp.dl_vec4 != 0;   // rows start on 16-byte boundaries only then
-    for (int bm = warp; bm < (fp.sample_only ? 0 : BM); bm += 4) {
+    for (int bm = warp; bm < (kSampleOnly ? 0 : BM); bm += 4) {
       const float* row = cp.draft_logits + (size_t)bm * V;
       float m = -INFINITY, s = 0.f;
       if (vec4) {
@@ -434,7 +441,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         if (x >= v_lo && x < v_hi) ws.qgath[bm] = __ldcg(row + x);
       }
     }
-    for (int bm = cta * 4 + warp; bm < (fp.sample_only ? 0 : BM); bm += G * 4) {
+    for (int bm = cta * 4 + warp; bm < (kSampleOnly ? 0 : BM); bm += G * 4) {
       const int b = bm / M, j = bm % M;
       const uint4* h4 = reinterpret_cast<const uint4*>(H + ((size_t)b * (M + 1) + j + 1) * cp.d);
       const uint4* w4 = reinterpret_cast<const uint4*>(wj);
@@ -459,7 +466,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     // starts when the whole accumulation is complete. A CTA that ran an early sweep (T_early > 0)
     // first takes, in phase 0, the statistics of the early tiles while the last sweep still streams,
     // and merges the two (max, sum exp) pairs per row at the end.
-    if (fp.sample_only) {
+    if constexpr (kSampleOnly) {
       // an earlier kernel made the decisions; fetch what the token draw needs
       if (tid < cp.B) {
         ms.sel_row[tid] = ws.sel_row[tid];
@@ -476,11 +483,11 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       tc_fence_after();
       ok = ok && (*abort_flag == 0);
       const int i_lo = ph == 0 ? 0 : T_early, i_hi = ph == 0 ? T_early : T;
-      if (fp.sample_only) {
+      if constexpr (kSampleOnly) {
         // (h) mass of the sampling weights of each selected row over the phase's tiles.
         // Sample-only mode: every TMEM column is a selected row, so the tiles are read 16 columns
         // (= 16 sequences) at a time, like the statistics passes.
-        if (ok && cp.rule != JD_RULE_TOPK) {
+        if (ok) {
 #pragma unroll
           for (int c0 = 0; c0 < N_PAD; c0 += 16) {
             if (c0 >= cp.B) break;
@@ -632,7 +639,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
       epi_sync();
     }
-    if (!fp.sample_only) {
+    if constexpr (!kSampleOnly) {
     if (ok && cp.logits_debug != nullptr)
       dump_logits<N_PAD>(cp.logits_debug, T, t0, R, V, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0]);
     __threadfence();
@@ -652,7 +659,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     // the drafted token (its logit is known grid-wide since barrier 1) and note the lowest token id
     // that attains this CTA's row maximum. Counts go to global counters with integer atomics
     // (order-independent), the argmax candidates beside the per-CTA maxima.
-    if (ok && cp.rule == JD_RULE_TOPK) {
+    if (kTopK && ok) {
       int* wcnt = reinterpret_cast<int*>(&ms.wmax[0][0]);   // the float statistics have been written out
       int* widx = reinterpret_cast<int*>(&ms.wsum[0][0]);
 #pragma unroll
@@ -775,7 +782,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
     // top-K rule: the next token is the argmax of the selected row; CTA 0 folds the per-CTA maxima
     // and their candidates (larger value first, then lower token id). Nothing is drawn.
-    const bool draw = (cp.rule != JD_RULE_TOPK);
+    constexpr bool draw = !kTopK;
     if (ok && !draw && cta == 0) {
       for (int b = warp; b < cp.B; b += 4) {
         const int row = ms.sel_row[b];
@@ -804,7 +811,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     // done above, phase by phase, as the tiles completed).
     // Full mode: the few selected rows sit in scattered columns; four sequences at a time so
     // that their draft-logit loads are in flight together.
-    if (ok && draw && !fp.sample_only) {
+    if (ok && draw && !kSampleOnly) {
       for (int b0 = 0; b0 < cp.B; b0 += 4) {
         double sr[4] = {0.0, 0.0, 0.0, 0.0}, sp[4] = {0.0, 0.0, 0.0, 0.0};
         for (int i0 = 0; i0 < T; i0 += 8) {
@@ -825,7 +832,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           for (int q = 0; q < 4; ++q) {
             if (b0 + q >= cp.B) continue;   // uniform over the CTA: no work for sequences that do not exist
             const int b = b0 + q;
-            const int col = fp.sample_only ? b : ms.sel_row[b];   // TMEM column of this sequence's selected row
+            const int col = kSampleOnly ? b : ms.sel_row[b];   // TMEM column of this sequence's selected row
             load_cols8<N_PAD>(i0, T, col, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale[col], &ms.swt[0][0], lg[q]);
           }
 #pragma unroll
@@ -948,7 +955,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       for (int b = 0; b < cp.B; ++b) {
         if (ms.own_cta[b] != cta) continue;
         const int row = ms.sel_row[b];
-        const int col = fp.sample_only ? b : row;
+        const int col = kSampleOnly ? b : row;
         const int kind = ms.own_usep[b] ? 1 : ms.sel_kind[b];
         const float lse_p = ms.sel_lse_p[b], lse_q = ms.sel_lse_q[b];
         const float* dlrow = cp.draft_logits + ((size_t)b * M + (row % (M + 1))) * V;
@@ -961,7 +968,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
           for (int u = 0; u < 8; ++u) {
             const int vg = (t0 + i0 + u) * kVocabTile + tid;
-            const float* src = fp.sample_only ? ws.w_sel + ((size_t)(t0 + i0 + u) * cp.B + b) * kVocabTile + tid
+            const float* src = kSampleOnly ? ws.w_sel + ((size_t)(t0 + i0 + u) * cp.B + b) * kVocabTile + tid
                                               : dlrow + vg;
             dv[u] = (kind == 0 && i0 + u < T && vg < V) ? __ldcg(src) : 0.f;
           }
@@ -1039,11 +1046,11 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   }
 }
 
-template <int N_PAD, bool kFp8>
+template <int N_PAD, bool kFp8, int kKind>
 cudaError_t launch_fused(const CUtensorMap& tmW, const CUtensorMap& tmH, const CallParams& cp, const Workspace& ws,
                          const void* H, const void* wj, const float* w_scale, const FusedParams& fp,
                          const FusedPlan& plan, cudaStream_t st) {
-  auto kern = fused_verify_kernel<N_PAD, kFp8>;   // its shared-memory limit was raised by fused_configure()
+  auto kern = fused_verify_kernel<N_PAD, kFp8, kKind>;   // its shared-memory limit was raised by fused_configure()
   const __nv_bfloat16* Hp = (const __nv_bfloat16*)H;
   const __nv_bfloat16* wp = (const __nv_bfloat16*)wj;
   void* args[] = {(void*)&tmW, (void*)&tmH, (void*)&cp, (void*)&ws, (void*)&Hp, (void*)&wp, (void*)&w_scale, (void*)&fp};
@@ -1068,12 +1075,28 @@ void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st) 
 }
 
 namespace {
+template <int N_PAD, bool kFp8>
+bool configure_kinds() {
+  return cudaFuncSetAttribute(fused_verify_kernel<N_PAD, kFp8, kFullSampling>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess &&
+         cudaFuncSetAttribute(fused_verify_kernel<N_PAD, kFp8, kFullTopK>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess &&
+         cudaFuncSetAttribute(fused_verify_kernel<N_PAD, kFp8, kSampleOnlyKind>,
+                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem) == cudaSuccess;
+}
 template <int N_PAD>
-bool configure_pair() {
-  return cudaFuncSetAttribute(fused_verify_kernel<N_PAD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              kMaxDynamicSmem) == cudaSuccess &&
-         cudaFuncSetAttribute(fused_verify_kernel<N_PAD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              kMaxDynamicSmem) == cudaSuccess;
+bool configure_pair() { return configure_kinds<N_PAD, false>() && configure_kinds<N_PAD, true>(); }
+
+template <int N_PAD>
+cudaError_t launch_n(bool fp8, int kind, const CUtensorMap& tmW, const CUtensorMap& tmH, const CallParams& cp,
+                     const Workspace& ws, const void* H, const void* wj, const float* w_scale, const FusedParams& fp,
+                     const FusedPlan& plan, cudaStream_t st) {
+#define JD_LAUNCH(FP8, KIND) launch_fused<N_PAD, FP8, KIND>(tmW, tmH, cp, ws, H, wj, w_scale, fp, plan, st)
+  if (fp8) return kind == kSampleOnlyKind ? JD_LAUNCH(true, kSampleOnlyKind)
+                                          : (kind == kFullTopK ? JD_LAUNCH(true, kFullTopK) : JD_LAUNCH(true, kFullSampling));
+  return kind == kSampleOnlyKind ? JD_LAUNCH(false, kSampleOnlyKind)
+                                 : (kind == kFullTopK ? JD_LAUNCH(false, kFullTopK) : JD_LAUNCH(false, kFullSampling));
+#undef JD_LAUNCH
 }
 }  // namespace
 
@@ -1139,7 +1162,6 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
   fp.tmem_tiles = plan.tmem_tiles;
   fp.tile_stride = plan.tile_stride;
   fp.R = sample_only ? cp.B : cp.B * (cp.M + 1);
-  fp.sample_only = sample_only ? 1 : 0;
   // Early sweep + one late tile: measured on B200 over 16 to 80 padded rows and d = 4096 to 16384,
   // it shortens the call by 2-4 % once the statistics passes are long enough to be worth hiding
   // (48 padded rows or more, or 32 with at least 128 k-steps) and lengthens it by 1-5 % below that.
@@ -1152,20 +1174,16 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
   const int n_ovf = plan.max_tiles - plan.tmem_tiles;
   fp.off_w = fp.off_ovf + (uint32_t)n_ovf * kVocabTile * plan.n_pad * 4;
   fp.off_w = (fp.off_w + 1023u) & ~1023u;
+  const int kind = sample_only ? kSampleOnlyKind : (cp.rule == JD_RULE_TOPK ? kFullTopK : kFullSampling);
+  const bool f8 = fp.fp8 != 0;
   cudaError_t e;
   switch (plan.n_pad) {
-    case 16: e = fp.fp8 ? launch_fused<16, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
-                       : launch_fused<16, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 32: e = fp.fp8 ? launch_fused<32, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
-                       : launch_fused<32, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 48: e = fp.fp8 ? launch_fused<48, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
-                       : launch_fused<48, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 64: e = fp.fp8 ? launch_fused<64, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
-                       : launch_fused<64, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 80: e = fp.fp8 ? launch_fused<80, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
-                       : launch_fused<80, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
-    case 96: e = fp.fp8 ? launch_fused<96, true>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st)
-                       : launch_fused<96, false>(tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 16: e = launch_n<16>(f8, kind, tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 32: e = launch_n<32>(f8, kind, tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 48: e = launch_n<48>(f8, kind, tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 64: e = launch_n<64>(f8, kind, tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 80: e = launch_n<80>(f8, kind, tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
+    case 96: e = launch_n<96>(f8, kind, tmW, tmH, cp, ws, H, w_judge, w_scale_fp8, fp, plan, st); break;
     default: e = cudaErrorInvalidValue; break;
   }
   *err = e;

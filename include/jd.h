@@ -194,8 +194,14 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* args, void* cuda_st
  * logits_debug must be NULL. */
 jd_status_t jd_verify_host(jd_handle_t h, const jd_verify_args_t* args, void* cuda_stream);
 
-/* Synchronises the stream of the handle's last jd_verify and copies the device status word:
- * *out = JD_OK, JD_ERR_TIMEOUT or JD_ERR_BAD_TOKEN. */
+/* Synchronises the stream of the handle's last jd_verify and reads the device status of that call:
+ * *out = JD_OK, JD_ERR_TIMEOUT or JD_ERR_BAD_TOKEN. Consecutive calls of the fused variant enqueue
+ * no memset between them (the kernel keeps its grid-barrier counters clean and tags its status
+ * writes with a launch number, so a clamped token of an earlier call is not reported for a later
+ * one). JD_ERR_TIMEOUT is different: a call in which a wait ran out leaves those counters in an
+ * unknown state, so every later fused call on the handle gives up at once and reports
+ * JD_ERR_TIMEOUT too, until this function has been called; the next jd_verify then starts from a
+ * cleared block. */
 jd_status_t jd_last_device_status(jd_handle_t h, int* out);
 
 /* Test helper for the failure path: launches a two-CTA kernel whose barrier wait can never be

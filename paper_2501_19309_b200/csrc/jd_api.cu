@@ -33,6 +33,7 @@ struct jd_handle_s {
   SideStream side;         // batched variant: draft statistics run next to the GEMM
   int last_variant;
   int last_launches;
+  bool needs_clear;        // the status / barrier block must be cleared by the host before the next launch
   // device staging of the host-buffer entry point (allocated on first use)
   void* st_H;
   int32_t* st_x;
@@ -373,8 +374,13 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
   if (variant == JD_VARIANT_BATCHED && !batched_ok) return JD_ERR_UNSUPPORTED;
 
   if (cudaSetDevice(c.device) != cudaSuccess) return JD_ERR_CUDA;
-  // status word and the grid-barrier counters behind it start every call at zero
-  if (cudaMemsetAsync(h->ws.status, 0, 512, st) != cudaSuccess) return JD_ERR_CUDA;
+  // Status word and barrier block. The fused kernel keeps them clean across its own launches, so a fused call
+  // that follows a fused call enqueues no memset; anything else (another variant before or now, an uncleared
+  // timeout, the handle's first call) starts from zeroes.
+  if (variant != JD_VARIANT_FUSED || h->last_variant != JD_VARIANT_FUSED || h->needs_clear) {
+    if (cudaMemsetAsync(h->ws.status, 0, 512, st) != cudaSuccess) return JD_ERR_CUDA;
+    h->needs_clear = false;
+  }
   if (a->rule == JD_RULE_TOPK) {   // rank counters start at zero, argmax candidates at a large id
     if (cudaMemsetAsync(h->ws.cnt, 0, (size_t)R * 4, st) != cudaSuccess ||
         cudaMemsetAsync(h->ws.argidx, 0x7F, (size_t)R * 4, st) != cudaSuccess)
@@ -525,9 +531,16 @@ jd_status_t jd_last_device_status(jd_handle_t h, int* out) {
   if (!h || !out) return JD_ERR_INVALID_ARG;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return JD_ERR_CUDA;
   if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return JD_ERR_CUDA;
-  unsigned s = 0;
-  if (cudaMemcpy(&s, h->ws.status, sizeof(s), cudaMemcpyDeviceToHost) != cudaSuccess) return JD_ERR_CUDA;
-  *out = (int)s;
+  // status word and, 256 bytes on, the barrier block with the fused kernel's launch counter
+  unsigned blk[64 + kCallCounter + 1];
+  if (cudaMemcpy(blk, h->ws.status, sizeof(blk), cudaMemcpyDeviceToHost) != cudaSuccess) return JD_ERR_CUDA;
+  const unsigned word = blk[0], done = blk[64 + kCallCounter];
+  const unsigned tag = word >> 8, code = word & 0xFFu;
+  // untagged: written since the host last cleared the block; tagged: by the last launch that finished
+  // (tag == done) or by one that gave up (tag == done + 1). Older tags belong to earlier calls.
+  const bool current = tag == 0u || tag == (done & 0xFFFFFFu) || tag == ((done + 1u) & 0xFFFFFFu);   // tags are 24 bits
+  *out = current ? (int)code : (int)JD_OK;
+  if (*out == JD_ERR_TIMEOUT) h->needs_clear = true;   // the counters of a launch that gave up are in an unknown state
   return JD_OK;
 }
 
@@ -538,6 +551,7 @@ jd_status_t jd_selftest_timeout(jd_handle_t h, uint32_t spin_limit, void* cuda_s
   if (cudaMemsetAsync(h->ws.status, 0, 512, st) != cudaSuccess) return JD_ERR_CUDA;
   launch_timeout_probe(h->ws, spin_limit, st);
   if (cudaGetLastError() != cudaSuccess) return JD_ERR_CUDA;
+  h->needs_clear = true;
   h->last_stream = st;
   return JD_OK;
 }

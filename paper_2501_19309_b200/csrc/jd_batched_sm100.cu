@@ -358,7 +358,6 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
     cc.next_token = cp.next_token + off;
     Workspace wc = ws;
     wc.sel_row += off; wc.sel_kind += off; wc.sel_lse_p += off; wc.sel_lse_q += off; wc.sel_u += off;
-    if (off > 0 && (*err = cudaMemsetAsync(ws.barrier, 0, 256, st)) != cudaSuccess) return -1;   // grid barriers restart
     // second pass operand: the bf16 rows, or their E4M3 codes (one byte per element)
     gather_rows_kernel<<<dim3(nc, 32), 256, 0, st>>>(cc, wc, fp8 ? ws.h8 : (const uint8_t*)H, fp8 ? cp.d : cp.d * 2);
     FusedPlan plan;

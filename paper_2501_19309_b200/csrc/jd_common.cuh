@@ -46,13 +46,36 @@ struct Workspace {
   int* argidx;         // [maxR] top-K rule: lowest token id that attains the row maximum
   int* part_idx;       // [maxR][np] top-K rule, fused variant: per-CTA argmax candidates
   __nv_bfloat16* h_sel;  // [maxB][d] selected rows of H gathered for the batched variant's second pass
-  unsigned* status;    // [1] device status word (jd_status_t of the first device-side problem)
-  unsigned* barrier;   // [8] grid-barrier counters of the fused variant
+  unsigned* status;    // [1] device status word: jd_status_t of the first device-side problem in bits 0-7; bits 8-31 a
+                       //     call tag when the fused kernel wrote it (see kCallCounter), 0 when another kernel did
+  unsigned* barrier;   // [8] fused variant: two sets of three grid-barrier counters ([0..2], [3..5]) used by
+                       //     alternate launches, [6] = kCallCounter, [7] the self-test's counter
   int np_cap;          // capacity (partials per row) of part_* and mass_*
   int nq_cap;          // capacity of qpart_*
 };
 
 __device__ __forceinline__ void set_status(unsigned* status, unsigned code) { atomicCAS(status, 0u, code); }
+
+// The fused kernel keeps its grid-barrier state clean by itself, so that back-to-back calls need no
+// memset between them. barrier[kCallCounter] counts the kernel's successful launches since the block
+// was last cleared by the host. Launch number c (0-based) uses barrier set c % 2, clears the other
+// set (idle since launch c - 1 ended) and, when it has passed its last barrier, CTA 0 publishes c + 1.
+// Its status writes carry the tag c + 1, which tells them apart from what earlier launches left in
+// the word. A launch in which a wait ran out publishes nothing: the next launch finds that tagged
+// JD_ERR_TIMEOUT still in place and gives up at once, and so on until the host has read the status
+// and cleared the block (the counters of the failed launch are in an unknown state).
+constexpr int kCallCounter = 6;
+__device__ __forceinline__ unsigned load_volatile_u32(const unsigned* p) { return *reinterpret_cast<const volatile unsigned*>(p); }
+__device__ __forceinline__ void set_status_tagged(unsigned* status, unsigned tag, unsigned code) {
+  const unsigned want = (tag << 8) | code;
+  unsigned old = load_volatile_u32(status);
+  for (int i = 0; i < 64; ++i) {                          // first problem of this launch wins
+    if ((old >> 8) == tag && (old & 0xFFu) != 0u) return;
+    const unsigned prev = atomicCAS(status, old, want);
+    if (prev == old) return;
+    old = prev;
+  }
+}
 
 // ---------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0, k1), ten rounds of

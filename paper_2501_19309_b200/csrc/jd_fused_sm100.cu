@@ -65,6 +65,8 @@ struct FusedParams {
   // the epilogue warps wait for it (bounded) before their first read of the draft logits.
   const unsigned* dl_flag;
   unsigned dl_epoch;
+  int plain_status; // 1: the caller clears status word and barrier block before every launch and wants plain codes
+                    //    in the word (no call tag)
   uint32_t off_h;   // byte offsets inside dynamic smem (from the 1024-aligned base)
   uint32_t off_ovf;
   uint32_t off_w;
@@ -80,6 +82,8 @@ struct Misc {
   uint32_t tmem_base;
   int abort_flag;
   int glist_n;              // rows whose drafted token lies in this CTA's vocabulary slice
+  unsigned launch_index;    // barrier[kCallCounter] at the start of this launch
+  int give_up;              // 1: an earlier launch's timeout has not been cleared by the host yet
   float wmax[4][N_PAD];
   float wsum[4][N_PAD];
   float cta_max[N_PAD];
@@ -215,6 +219,12 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const int n_ovf = max(0, T - fp.tmem_tiles);   // first n_ovf tiles go through TMEM into smem
   const int R = fp.R, M = cp.M, V = cp.V;
   const int BM = cp.B * M;
+  // device-side problems go to the status word, tagged with this launch's number unless the caller
+  // clears the word before every launch (the counter does not move while a launch can still report)
+  auto report = [&](unsigned code) {
+    if (fp.plain_status) set_status(ws.status, code);
+    else set_status_tagged(ws.status, load_volatile_u32(ws.barrier + kCallCounter) + 1u, code);
+  };
 
   // The producer warp sets up the barriers and leaves the prologue without waiting for the other
   // warps (it arrives at the block's hand-over barrier, they wait on it), so that W starts to
@@ -229,13 +239,18 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     ms.glist_n = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (tid == 0) {
+    const unsigned c = fp.plain_status ? 0u : load_volatile_u32(ws.barrier + kCallCounter);
+    ms.launch_index = c;
+    ms.give_up = (!fp.plain_status && load_volatile_u32(ws.status) == (((c + 1u) << 8) | (unsigned)JD_ERR_TIMEOUT)) ? 1 : 0;
+  }
   if (tid < N_PAD) {
     int x = -1;
     if (tid < R && !kSampleOnly) {
       const int b = tid / (M + 1), j = tid % (M + 1);
       if (j < M) {
         x = cp.draft_tokens[b * M + j];
-        if (x < 0 || x >= V) { set_status(ws.status, JD_ERR_BAD_TOKEN); x = min(max(x, 0), V - 1); }
+        if (x < 0 || x >= V) { report(JD_ERR_BAD_TOKEN); x = min(max(x, 0), V - 1); }
       }
     }
     ms.x_row[tid] = x;
@@ -305,7 +320,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
       }
     }
-    if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
+    if (!ok) report(JD_ERR_TIMEOUT);
   } else if (warp == 5 && lane == 0) {
     // ------------------------------------------------------------------ MMA issuer
     const uint32_t idesc = kFp8 ? make_idesc_e4m3(N_PAD) : make_idesc(N_PAD);
@@ -345,12 +360,17 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
       if (ok) umma_commit(smem_u32(&ms.acc_full[g]));
     }
-    if (!ok) set_status(ws.status, JD_ERR_TIMEOUT);
+    if (!ok) report(JD_ERR_TIMEOUT);
   } else if (warp < 4) {
     // ------------------------------------------------------------------ epilogue warps
     const uint32_t tmem_lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
     const int ts = fp.tile_stride;
+    unsigned* const bar = ws.barrier + (ms.launch_index & 1u) * 3u;   // this launch's set of barrier counters
     bool ok = true;
+    if (ms.give_up) {   // an uncleared timeout of an earlier launch: every role leaves through the failure path
+      ok = false;
+      if (tid == 0) *abort_flag = 1;
+    }
 
     // (a) overflow tiles: TMEM -> smem as soon as their accumulation is complete
     if (n_ovf > 0) {
@@ -390,7 +410,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
         if (!arrived) {
           *abort_flag = 1;
-          set_status(ws.status, JD_ERR_TIMEOUT);
+          report(JD_ERR_TIMEOUT);
         }
       }
       epi_sync();
@@ -647,9 +667,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
     // ------------------------------------------------------------------ grid barrier 1
     if (tid == 0) {
-      if (!ok || !grid_arrive_and_wait(ws.barrier + 0, (unsigned)G, abort_flag)) {
+      if (!ok || !grid_arrive_and_wait(bar + 0, (unsigned)G, abort_flag)) {
         *abort_flag = 1;
-        set_status(ws.status, JD_ERR_TIMEOUT);
+        report(JD_ERR_TIMEOUT);
       }
     }
     epi_sync();
@@ -750,9 +770,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
     // ------------------------------------------------------------------ grid barrier 2
     if (tid == 0) {
-      if (!ok || !grid_arrive_and_wait(ws.barrier + 1, (unsigned)G, abort_flag)) {
+      if (!ok || !grid_arrive_and_wait(bar + 1, (unsigned)G, abort_flag)) {
         *abort_flag = 1;
-        set_status(ws.status, JD_ERR_TIMEOUT);
+        report(JD_ERR_TIMEOUT);
       }
     }
     epi_sync();
@@ -870,9 +890,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
     // ------------------------------------------------------------------ grid barrier 3
     if (tid == 0 && draw) {
-      if (!ok || !grid_arrive_and_wait(ws.barrier + 2, (unsigned)G, abort_flag)) {
+      if (!ok || !grid_arrive_and_wait(bar + 2, (unsigned)G, abort_flag)) {
         *abort_flag = 1;
-        set_status(ws.status, JD_ERR_TIMEOUT);
+        report(JD_ERR_TIMEOUT);
       }
     }
     epi_sync();
@@ -1029,6 +1049,14 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         if (tid == 0) cp.next_token[b] = token < 0 ? 0 : token;
       }
     }
+    // Every barrier of this launch lies behind CTA 0 now and nothing can report any more: clear the set
+    // the previous launch used and publish this launch as done (the next one then takes that set).
+    if (!fp.plain_status && cta == 0 && tid == 0 && ok) {
+      unsigned* other = ws.barrier + ((ms.launch_index & 1u) ^ 1u) * 3u;
+      other[0] = 0u; other[1] = 0u; other[2] = 0u;
+      __threadfence();
+      *reinterpret_cast<volatile unsigned*>(ws.barrier + kCallCounter) = ms.launch_index + 1u;
+    }
     tc_fence_before();
   }
 
@@ -1150,8 +1178,10 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
 
 int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
               const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err,
-              bool sample_only, const float* w_scale_fp8, const unsigned* dl_flag, unsigned dl_epoch) {
+              bool sample_only, const float* w_scale_fp8, const unsigned* dl_flag, unsigned dl_epoch,
+              bool plain_status) {
   FusedParams fp;
+  fp.plain_status = plain_status ? 1 : 0;
   fp.dl_flag = sample_only ? nullptr : dl_flag;
   fp.dl_epoch = dl_epoch;
   fp.fp8 = w_scale_fp8 ? 1 : 0;

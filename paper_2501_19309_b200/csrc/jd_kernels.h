@@ -43,10 +43,12 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
 // Returns the number of kernels launched, or -1 with *err set. dl_flag (optional): a device word
 // that another stream sets to dl_epoch once the draft logits have been copied in; the kernel then
 // starts streaming W at once and waits for the word before it first reads the draft logits.
+// plain_status: the caller clears ws.status and ws.barrier before every launch and wants untagged status
+// codes; otherwise the kernel keeps the barrier block clean across launches by itself (jd_common.cuh).
 int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW, const CUtensorMap& tmH,
               const void* H, const void* w_judge, const FusedPlan& plan, cudaStream_t st, cudaError_t* err,
               bool sample_only = false, const float* w_scale_fp8 = nullptr, const unsigned* dl_flag = nullptr,
-              unsigned dl_epoch = 0);
+              unsigned dl_epoch = 0, bool plain_status = false);
 
 // Two-pass tensor-core variant for many rows (jd_batched_sm100.cu). tmW256 / tmW128: W with
 // 256- and 128-row boxes; tmH: H with a 128-row box; tmHsel: the handle's [B, d] gather buffer

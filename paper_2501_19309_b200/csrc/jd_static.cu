@@ -165,7 +165,7 @@ extern "C" jd_status_t jd_verify_static(int32_t d, int32_t V, const void* W, con
   if (cudaMemsetAsync(own_status, 0, 512, st) != cudaSuccess) return JD_ERR_CUDA;
   if (device_status && cudaMemsetAsync(device_status, 0, sizeof(uint32_t), st) != cudaSuccess) return JD_ERR_CUDA;
   cudaError_t err = cudaSuccess;
-  if (run_fused(cp, ws, tm_w, tm_h, a->H, w_judge, plan, st, &err) < 0) {
+  if (run_fused(cp, ws, tm_w, tm_h, a->H, w_judge, plan, st, &err, false, nullptr, nullptr, 0, /*plain_status=*/true) < 0) {
     cudaGetLastError();
     return JD_ERR_CUDA;
   }

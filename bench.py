@@ -80,6 +80,7 @@ def record_traffic(csv_specs) -> None:
     dram__bytes_read.sum / dram__bytes_write.sum columns. The bytes of the first captured launch of
     each file are added up per workload (a workload whose call runs two kernels gives two files)."""
     import csv
+    import re
     out = {"kernel_source_sha256_16": kernel_source_hash(), "workloads": {},
            "note": "dram__bytes_read.sum + dram__bytes_write.sum of one launch of each dominant kernel"}
     scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
@@ -91,7 +92,9 @@ def record_traffic(csv_specs) -> None:
                 rows = [r for r in csv.reader(f) if r]
             hdr = next(i for i, r in enumerate(rows) if "Kernel Name" in r)
             cols, units, first = rows[hdr], rows[hdr + 1], rows[hdr + 2]
-            kernels.append(first[cols.index("Kernel Name")].split("(")[0])
+            name = first[cols.index("Kernel Name")]
+            m = re.search(r"(\w+<[^>]*>)", name)
+            kernels.append(m.group(1) if m else name.split("(")[0])
             for m in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
                 i = cols.index(m)
                 total += float(first[i].replace(",", "")) * scale[units[i]]

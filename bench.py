@@ -92,9 +92,9 @@ def record_traffic(csv_specs) -> None:
                 rows = [r for r in csv.reader(f) if r]
             hdr = next(i for i, r in enumerate(rows) if "Kernel Name" in r)
             cols, units, first = rows[hdr], rows[hdr + 1], rows[hdr + 2]
-            name = first[cols.index("Kernel Name")]
-            m = re.search(r"(\w+<[^>]*>)", name)
-            kernels.append(m.group(1) if m else name.split("(")[0])
+            kname = first[cols.index("Kernel Name")]
+            m = re.search(r"(\w+<[^>]*>)", kname)
+            kernels.append(m.group(1) if m else kname.split("(")[0])
             for m in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
                 i = cols.index(m)
                 total += float(first[i].replace(",", "")) * scale[units[i]]

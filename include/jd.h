@@ -211,6 +211,13 @@ jd_status_t jd_last_device_status(jd_handle_t h, int* out);
  * same way (limit 2^22). */
 jd_status_t jd_selftest_timeout(jd_handle_t h, uint32_t spin_limit, void* cuda_stream);
 
+/* Test helper for the fail-stop rule described at jd_last_device_status: marks the handle's device
+ * status as a fused call that gave up would have left it (nothing waits, nothing runs out, the host
+ * side of the handle is not told). A fused jd_verify enqueued afterwards must return at once with
+ * device status JD_ERR_TIMEOUT, and the first call after jd_last_device_status has reported it must
+ * run normally again. */
+jd_status_t jd_selftest_stale_timeout(jd_handle_t h, void* cuda_stream);
+
 /* Variant the last jd_verify on this handle ran (jd_variant_t), 0 before the first call, and
  * the number of kernels it launched. Either pointer may be NULL. */
 jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launches);

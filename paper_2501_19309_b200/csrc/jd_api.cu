@@ -556,6 +556,15 @@ jd_status_t jd_selftest_timeout(jd_handle_t h, uint32_t spin_limit, void* cuda_s
   return JD_OK;
 }
 
+jd_status_t jd_selftest_stale_timeout(jd_handle_t h, void* cuda_stream) {
+  if (!h) return JD_ERR_INVALID_ARG;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return JD_ERR_CUDA;
+  launch_stale_timeout(h->ws, (cudaStream_t)cuda_stream);
+  if (cudaGetLastError() != cudaSuccess) return JD_ERR_CUDA;
+  h->last_stream = (cudaStream_t)cuda_stream;
+  return JD_OK;   // on purpose not remembered on the host: the device-side rule is what is being tested
+}
+
 jd_status_t jd_stream_read_probe(const void* data, size_t bytes, uint32_t* out, void* cuda_stream) {
   if (!data || !out || bytes < 16 || !aligned16(data)) return JD_ERR_INVALID_ARG;
   int dev = 0, sms = 0;

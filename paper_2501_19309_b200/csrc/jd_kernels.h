@@ -39,6 +39,7 @@ constexpr int kMaxDynamicSmem = 227 * 1024;
 bool fused_configure();
 bool batched_configure();
 void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st);
+void launch_stale_timeout(const Workspace& ws, cudaStream_t st);
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan);
 // Returns the number of kernels launched, or -1 with *err set. dl_flag (optional): a device word
 // that another stream sets to dl_epoch once the draft logits have been copied in; the kernel then

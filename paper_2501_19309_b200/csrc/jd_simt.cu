@@ -485,9 +485,18 @@ __global__ void __launch_bounds__(512) stream_read_kernel(const uint4* __restric
   if ((threadIdx.x & 31) == 0 && acc != 0) atomicXor(out, acc);
 }
 
+// Self-test of the fused variant's fail-stop rule: leaves the status word as a fused launch that gave up
+// would (a timeout tagged with the number of the next launch), without any wait having run out.
+__global__ void stale_timeout_kernel(Workspace ws) {
+  if (threadIdx.x == 0)
+    set_status_tagged(ws.status, load_volatile_u32(ws.barrier + kCallCounter) + 1u, JD_ERR_TIMEOUT);
+}
+
 // -----------------------------------------------------------------------------------------
 // host-side launchers
 // -----------------------------------------------------------------------------------------
+void launch_stale_timeout(const Workspace& ws, cudaStream_t st) { stale_timeout_kernel<<<1, 32, 0, st>>>(ws); }
+
 int launch_q_stats(const CallParams& cp, const Workspace& ws, cudaStream_t st) {
   const int nq = (cp.V + kQChunk - 1) / kQChunk;
   q_stats_kernel<<<dim3(nq, cp.B * cp.M), 256, 0, st>>>(cp, ws, nq);

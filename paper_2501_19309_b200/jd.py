@@ -34,7 +34,7 @@ VARIANTS = {"auto": JD_VARIANT_AUTO, "simt": JD_VARIANT_SIMT, "fused": JD_VARIAN
 EXPORTS = ["jd_version", "jd_status_string", "jd_workspace_bytes", "jd_create", "jd_destroy", "jd_set_head",
            "jd_verify", "jd_verify_host", "jd_last_device_status", "jd_last_launch_info", "jd_philox_uniforms",
            "jd_verify_static", "jd_set_head_fp8", "jd_selftest_timeout", "jd_stream_read_probe",
-           "jd_quantize_rows_e4m3", "jd_check_workspace_guards"]
+           "jd_quantize_rows_e4m3", "jd_check_workspace_guards", "jd_selftest_stale_timeout"]
 
 
 class jd_config_t(C.Structure):
@@ -91,6 +91,7 @@ def load():
                                      C.POINTER(jd_verify_args_t), C.c_void_p, C.c_void_p]
     lib.jd_quantize_rows_e4m3.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.jd_check_workspace_guards.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+    lib.jd_selftest_stale_timeout.argtypes = [C.c_void_p, C.c_void_p]
     for name in EXPORTS:
         if name not in ("jd_version", "jd_status_string", "jd_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -142,6 +143,10 @@ def jd_verify_host(h, args: jd_verify_args_t, stream_ptr: int = 0) -> int:
 
 def jd_selftest_timeout(h, spin_limit: int, stream_ptr: int = 0) -> int:
     return load().jd_selftest_timeout(h, C.c_uint32(spin_limit), C.c_void_p(stream_ptr))
+
+
+def jd_selftest_stale_timeout(h, stream_ptr: int = 0) -> int:
+    return load().jd_selftest_stale_timeout(h, C.c_void_p(stream_ptr))
 
 
 def jd_last_device_status(h) -> int:

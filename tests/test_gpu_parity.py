@@ -473,6 +473,39 @@ def test_bounded_wait_reports_timeout_and_handle_stays_usable():
     ver.close()
 
 
+@pytest.mark.parametrize("B,M,d,V", [(1, 8, 256, 128256), (4, 16, 128, 128256), (6, 15, 64, 128256)])
+def test_fused_calls_stop_after_an_uncleared_timeout_and_recover_once_it_was_read(B, M, d, V):
+    """Back-to-back fused calls share no memset: the kernel keeps its barrier counters clean and tags its
+    status writes. A call that gave up leaves the counters unknown, so every later call must give up at once
+    (device status JD_ERR_TIMEOUT, no wait runs its full limit) until the host has read the status; the call
+    after that starts from a cleared block and is correct again."""
+    import time
+    import torch
+    from paper_2501_19309_b200 import jd
+    wl = I.CONFIGS[2].scaled("stale-%d-%d-%d-%d" % (B, M, d, V), B=B, M=M, d=d, V=V)
+    inp = I.make_inputs(wl, 3)
+    dev = T.upload(inp)
+    ver = T.make_verifier(inp, dev)
+    ref = T.run_oracle(inp, "judge_or_standard", seed=0)
+    for _ in range(3):                                            # launches 0, 1, 2: both counter sets in use
+        got = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "judge_or_standard", variant="fused"))
+    assert ver.device_status() == jd.JD_OK
+    T.compare(got, ref, "judge_or_standard", M)
+    assert jd.jd_selftest_stale_timeout(ver.h, torch.cuda.current_stream().cuda_stream) == jd.JD_OK
+    t0 = time.perf_counter()
+    for _ in range(2):                                            # both give up at once
+        ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "judge_or_standard", variant="fused")
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0                         # nowhere near a wait's full limit
+    assert ver.device_status() == jd.JD_ERR_TIMEOUT               # read: the next call clears the block
+    for _ in range(2):
+        got = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "judge_or_standard", variant="fused"))
+        assert ver.device_status() == jd.JD_OK
+        T.compare(got, ref, "judge_or_standard", M)
+    assert ver.damaged_guards() == 0
+    ver.close()
+
+
 @pytest.mark.parametrize("B,M,d,V", [(1, 95, 64, 2000), (48, 1, 64, 5000), (1, 1, 64, 2), (2, 2, 64, 129)])
 def test_extreme_shapes(B, M, d, V):
     wl = I.CONFIGS[2].scaled("edge-%d-%d-%d-%d" % (B, M, d, V), B=B, M=M, d=d, V=V)

@@ -77,6 +77,7 @@ template <int N_PAD>
 struct Misc {
   uint64_t full_w[kMaxStages], empty_w[kMaxStages];
   uint64_t full_h[kMaxHStages], empty_h[kMaxHStages];
+  uint64_t full2[kMaxStages / 2], empty2[kMaxStages / 2];   // one-tile sweep: a pair of k-slices per barrier
   uint64_t acc_full[2];
   uint64_t drained;
   uint32_t tmem_base;
@@ -232,6 +233,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   if (warp == 4 && lane == 0) {
     for (int s = 0; s < fp.stages; ++s) { mbar_init(smem_u32(&ms.full_w[s]), 1); mbar_init(smem_u32(&ms.empty_w[s]), 1); }
     for (int s = 0; s < fp.h_stages; ++s) { mbar_init(smem_u32(&ms.full_h[s]), 1); mbar_init(smem_u32(&ms.empty_h[s]), 1); }
+    for (int s = 0; s < kMaxStages / 2; ++s) { mbar_init(smem_u32(&ms.full2[s]), 1); mbar_init(smem_u32(&ms.empty2[s]), 1); }
     mbar_init(smem_u32(&ms.acc_full[0]), 1);
     mbar_init(smem_u32(&ms.acc_full[1]), 1);
     mbar_init(smem_u32(&ms.drained), 1);
@@ -294,6 +296,13 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   const int g_begin[2] = {0, g_split};
   const int g_end[2] = {g_split, T};
   const uint32_t g_col[2] = {0u, (uint32_t)(T_early * fp.tile_stride)};   // first TMEM column of each group
+  // A sweep over a single tile is bound by what the MMA thread does per k-step (two waits, four MMAs, two
+  // commits: about 0.5 us for 16 KB of W), not by HBM. The one-tile late sweep therefore moves two k-slices
+  // of W and of H per barrier: ring slots 2s and 2s + 1 form a pair with barriers of its own, so that one
+  // wait and one commit serve eight MMAs. The pairs take over the slots once the first sweep has finished
+  // with all of them.
+  const int pairs = min(fp.stages, fp.h_stages) / 2;
+  const bool paired_late = T_early > 0 && T - T_early == 1 && (fp.num_kb & 1) == 0 && pairs >= 1;
 
   if (warp == 4 && lane == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -304,6 +313,26 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     bool ok = true;
     for (int g = 0; g < 2 && ok; ++g) {
       if (g_begin[g] == g_end[g]) continue;
+      if (g == 1 && paired_late) {
+        // every MMA of the first sweep has completed: all ring slots are free for the pairs
+        ok = mbar_wait(smem_u32(&ms.acc_full[0]), 0u, abort_flag);
+        int s2 = 0;
+        uint32_t ph2 = 0;
+        const int row0 = (t0 + g_begin[1]) * kVocabTile;
+        for (int kb = 0; kb < fp.num_kb && ok; kb += 2) {
+          ok = mbar_wait(smem_u32(&ms.empty2[s2]), ph2 ^ 1u, abort_flag);
+          if (!ok) break;
+          const uint32_t fb = smem_u32(&ms.full2[s2]);
+          mbar_expect_tx(fb, 2 * (kWStageBytes + N_PAD * 128));
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            tma_load_2d(sH + (2 * s2 + j) * (N_PAD * 128), &tmH, fb, (kb + j) * kelems, 0, pol_h);
+            tma_load_2d(sW + (2 * s2 + j) * kWStageBytes, &tmW, fb, (kb + j) * kelems, row0, pol_w);
+          }
+          if (++s2 == pairs) { s2 = 0; ph2 ^= 1u; }
+        }
+        continue;
+      }
       for (int kb = 0; kb < fp.num_kb && ok; ++kb) {
         ok = mbar_wait(smem_u32(&ms.empty_h[hs_i]), hph ^ 1u, abort_flag);
         if (!ok) break;
@@ -333,6 +362,31 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         ok = mbar_wait(smem_u32(&ms.drained), 0u, abort_flag);
         if (!ok) break;
         tc_fence_after();
+      }
+      if (g == 1 && paired_late) {
+        int s2 = 0;
+        uint32_t ph2 = 0;
+        const uint32_t dcol = tmem_base + g_col[1];
+        for (int kb = 0; kb < fp.num_kb && ok; kb += 2) {
+          ok = mbar_wait(smem_u32(&ms.full2[s2]), ph2, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint32_t wb = sW + (2 * s2 + j) * kWStageBytes, hb = sH + (2 * s2 + j) * (N_PAD * 128);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const uint64_t da = make_smem_desc(wb + k * 32), db = make_smem_desc(hb + k * 32);
+              const uint32_t acc = (kb > 0 || j > 0 || k > 0) ? 1u : 0u;
+              if constexpr (kFp8) umma_e4m3(dcol, da, db, idesc, acc);
+              else umma_bf16(dcol, da, db, idesc, acc);
+            }
+          }
+          umma_commit(smem_u32(&ms.empty2[s2]));
+          if (++s2 == pairs) { s2 = 0; ph2 ^= 1u; }
+        }
+        if (ok) umma_commit(smem_u32(&ms.acc_full[1]));
+        continue;
       }
       for (int kb = 0; kb < fp.num_kb && ok; ++kb) {
         ok = mbar_wait(smem_u32(&ms.full_h[hs_i]), hph, abort_flag);

@@ -303,6 +303,11 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   // with all of them.
   const int pairs = min(fp.stages, fp.h_stages) / 2;
   const bool paired_late = T_early > 0 && T - T_early == 1 && (fp.num_kb & 1) == 0 && pairs >= 1;
+  // The other sweeps, too, move two k-slices per ring slot whenever d allows it (kk = 2): one wait and one
+  // commit then serve eight MMAs of a tile instead of four, which keeps the producer and MMA threads'
+  // per-tile work safely below the time HBM needs for the tile's bytes.
+  const int kk = (fp.num_kb & 1) == 0 ? 2 : 1;
+  const int w_slots = fp.stages / kk, h_slots = fp.h_stages / kk;   // ring depths in slots of kk slices
 
   if (warp == 4 && lane == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -333,19 +338,21 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
         continue;
       }
-      for (int kb = 0; kb < fp.num_kb && ok; ++kb) {
+      for (int kb = 0; kb < fp.num_kb && ok; kb += kk) {
         ok = mbar_wait(smem_u32(&ms.empty_h[hs_i]), hph ^ 1u, abort_flag);
         if (!ok) break;
-        mbar_expect_tx(smem_u32(&ms.full_h[hs_i]), N_PAD * 128);
-        tma_load_2d(sH + hs_i * (N_PAD * 128), &tmH, smem_u32(&ms.full_h[hs_i]), kb * kelems, 0, pol_h);
-        if (++hs_i == fp.h_stages) { hs_i = 0; hph ^= 1u; }
+        mbar_expect_tx(smem_u32(&ms.full_h[hs_i]), kk * N_PAD * 128);
+        for (int j = 0; j < kk; ++j)
+          tma_load_2d(sH + (hs_i * kk + j) * (N_PAD * 128), &tmH, smem_u32(&ms.full_h[hs_i]), (kb + j) * kelems, 0, pol_h);
+        if (++hs_i == h_slots) { hs_i = 0; hph ^= 1u; }
         for (int i = g_begin[g]; i < g_end[g]; ++i) {
           ok = mbar_wait(smem_u32(&ms.empty_w[ws_i]), wph ^ 1u, abort_flag);
           if (!ok) break;
-          mbar_expect_tx(smem_u32(&ms.full_w[ws_i]), kWStageBytes);
-          tma_load_2d(sW + ws_i * kWStageBytes, &tmW, smem_u32(&ms.full_w[ws_i]), kb * kelems, (t0 + i) * kVocabTile,
-                      pol_w);
-          if (++ws_i == fp.stages) { ws_i = 0; wph ^= 1u; }
+          mbar_expect_tx(smem_u32(&ms.full_w[ws_i]), kk * kWStageBytes);
+          for (int j = 0; j < kk; ++j)
+            tma_load_2d(sW + (ws_i * kk + j) * kWStageBytes, &tmW, smem_u32(&ms.full_w[ws_i]), (kb + j) * kelems,
+                        (t0 + i) * kVocabTile, pol_w);
+          if (++ws_i == w_slots) { ws_i = 0; wph ^= 1u; }
         }
       }
     }
@@ -388,29 +395,30 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         if (ok) umma_commit(smem_u32(&ms.acc_full[1]));
         continue;
       }
-      for (int kb = 0; kb < fp.num_kb && ok; ++kb) {
+      for (int kb = 0; kb < fp.num_kb && ok; kb += kk) {
         ok = mbar_wait(smem_u32(&ms.full_h[hs_i]), hph, abort_flag);
         if (!ok) break;
-        const uint32_t hb = sH + hs_i * (N_PAD * 128);
         for (int i = g_begin[g]; i < g_end[g]; ++i) {
           ok = mbar_wait(smem_u32(&ms.full_w[ws_i]), wph, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t wb = sW + ws_i * kWStageBytes;
           const uint32_t dcol = tmem_base + g_col[g] + (uint32_t)((i - g_begin[g]) * fp.tile_stride);
+          for (int j = 0; j < kk; ++j) {
+            const uint32_t wb = sW + (ws_i * kk + j) * kWStageBytes, hb = sH + (hs_i * kk + j) * (N_PAD * 128);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {   // four MMAs of 32 bytes of K each: 16 bf16 or 32 FP8 codes
-            const uint64_t da = make_smem_desc(wb + k * 32), db = make_smem_desc(hb + k * 32);
-            const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-            if constexpr (kFp8) umma_e4m3(dcol, da, db, idesc, acc);
-            else umma_bf16(dcol, da, db, idesc, acc);
+            for (int k = 0; k < 4; ++k) {   // four MMAs of 32 bytes of K each: 16 bf16 or 32 FP8 codes
+              const uint64_t da = make_smem_desc(wb + k * 32), db = make_smem_desc(hb + k * 32);
+              const uint32_t acc = (kb > 0 || j > 0 || k > 0) ? 1u : 0u;
+              if constexpr (kFp8) umma_e4m3(dcol, da, db, idesc, acc);
+              else umma_bf16(dcol, da, db, idesc, acc);
+            }
           }
           umma_commit(smem_u32(&ms.empty_w[ws_i]));
-          if (++ws_i == fp.stages) { ws_i = 0; wph ^= 1u; }
+          if (++ws_i == w_slots) { ws_i = 0; wph ^= 1u; }
         }
         if (!ok) break;
         umma_commit(smem_u32(&ms.empty_h[hs_i]));
-        if (++hs_i == fp.h_stages) { hs_i = 0; hph ^= 1u; }
+        if (++hs_i == h_slots) { hs_i = 0; hph ^= 1u; }
       }
       if (ok) umma_commit(smem_u32(&ms.acc_full[g]));
     }

@@ -14,12 +14,16 @@
 //
 // Main loop, K-outer: for every 64-wide slice of d the H slice [N_PAD x 64] is loaded once and
 // multiplied with the W slice [128 x 64] of every tile of the group, so W streams from HBM
-// exactly once and H is re-read (from L2) once per group, not once per tile.
-// Where the statistics passes are long enough to matter (see run_fused), a CTA whose tiles all
-// fit in TMEM sweeps d twice: first over all tiles but the last, then over the last one. The
-// epilogue warps take the row statistics of the early tiles (in sample-only mode: their sampling
-// masses) while the last tile still streams, so only one tile's worth is left for the time after
-// the stream.
+// exactly once and H is re-read (from L2) once per group, not once per tile. A ring slot holds
+// two consecutive k-slices (when d / 64 is even), so that the single producer thread and the
+// single MMA thread spend one wait and one commit per eight MMAs: with one slice per slot their
+// per-tile work (about 0.36 us per 16 KB of W) was as long as HBM needs for those bytes, and longer
+// in a sweep over one tile.
+// Where it pays (see run_fused), a CTA whose tiles all fit in TMEM sweeps d twice: first over all
+// tiles but the last, then over the last one, that one with W and H of a pair of k-slices under a
+// single barrier. The epilogue warps take the row statistics of the early tiles (in sample-only
+// mode: their sampling masses) while the last tile still streams, so only one tile's worth is left
+// for the time after the stream.
 //
 // After the main loop the grid meets three times:
 //   per-CTA (max, sum exp) of every row, logit of the drafted tokens            -> barrier 1
@@ -46,6 +50,7 @@ constexpr int kTmemCols = 512;
 constexpr int kMiscBytes = 21504;                // barriers + reduction scratch at the head of smem
 constexpr int kMaxStages = 12;
 constexpr int kMinHStages = 4;
+constexpr int kPreferredHStages = 6;
 constexpr int kMaxHStages = 8;
 
 
@@ -1216,15 +1221,18 @@ bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* pla
   const size_t base_fixed = 1024 /*alignment slack*/ + kMiscBytes + (size_t)n_ovf * kVocabTile * n_pad * 4;
   const size_t h_stage = (size_t)n_pad * 128;
   const size_t budget = kMaxDynamicSmem;
-  size_t fixed = base_fixed + kMinHStages * h_stage;
-  if (fixed + 3 * (size_t)kWStageBytes > budget) return false;   // at least a three-deep W ring
-  int stages = (int)((budget - fixed) / kWStageBytes);
+  if (base_fixed + kMinHStages * h_stage + 3 * (size_t)kWStageBytes > budget) return false;   // at least a three-deep W ring
+  // Ring slots hold two k-slices, and the one-tile late sweep runs on min(W, H) / 2 pairs of them, so an H ring
+  // of four slices means two slots and two pairs in flight: measured 2-3 % slower per call than six or more
+  // (cfg1, cfg2, cfg3). Six H slices are set aside first wherever that still leaves a W ring of six.
+  int h_min = kPreferredHStages;
+  if (base_fixed + h_min * h_stage + 6 * (size_t)kWStageBytes > budget) h_min = kMinHStages;
+  int stages = (int)((budget - base_fixed - h_min * h_stage) / kWStageBytes);
   stages = std::min(stages, kMaxStages);
-  // The H ring takes whatever the W ring leaves over: a sweep over only one or two tiles per
-  // k-step can keep no more W stages in flight than (tiles per k-step) x (H stages).
+  // the H ring then takes whatever the W ring leaves over
   int h_stages = (int)((budget - base_fixed - (size_t)stages * kWStageBytes) / h_stage);
-  h_stages = std::max(kMinHStages, std::min(h_stages, kMaxHStages));
-  fixed = base_fixed + h_stages * h_stage;
+  h_stages = std::max(h_min, std::min(h_stages, kMaxHStages));
+  const size_t fixed = base_fixed + h_stages * h_stage;
   if (plan) {
     plan->num_ctas = num_sms;
     plan->n_pad = n_pad;
@@ -1254,13 +1262,12 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
   fp.tmem_tiles = plan.tmem_tiles;
   fp.tile_stride = plan.tile_stride;
   fp.R = sample_only ? cp.B : cp.B * (cp.M + 1);
-  // Early sweep + one late tile: measured on B200 over 16 to 80 padded rows and d = 4096 to 16384,
-  // it shortens the call by 2-4 % once the statistics passes are long enough to be worth hiding
-  // (48 padded rows or more, or 32 with at least 128 k-steps) and lengthens it by 1-5 % below that.
-  // In sample-only mode the early tiles' sampling masses are what the last sweep hides: 1-5 % shorter
-  // batched calls at 16 to 64 sequences.
-  fp.late_tiles = sample_only ? 1
-                              : ((plan.n_pad >= 48 || (plan.n_pad >= 32 && fp.num_kb >= 128)) ? 1 : 0);
+  // Early sweep + one late tile: the statistics of all tiles but the last (in sample-only mode: their sampling
+  // masses) are taken while the last tile streams. With the late sweep moving two k-slices per barrier it costs
+  // the stream nothing measurable, and per call it gains 3.5 % at 16 padded rows (d = 4096), about as much as
+  // before at 80 (cfg2) and is even with a single sweep at 32 rows and d = 16384 (cfg3): on wherever the sweep
+  // over d is long enough to hide something (32 k-steps) or the statistics passes are long (48 padded rows).
+  fp.late_tiles = (sample_only || plan.n_pad >= 48 || fp.num_kb >= 32) ? 1 : 0;
   fp.off_h = kMiscBytes;
   fp.off_ovf = fp.off_h + plan.h_stages * plan.n_pad * 128;
   const int n_ovf = plan.max_tiles - plan.tmem_tiles;

@@ -240,6 +240,8 @@ FUSED_SHAPES = [
     (4, 16, 128, 128256),     # 70B-head rows: n_pad 80, one tile per CTA overflows to shared memory
     (5, 15, 128, 128256 + 77),  # same with a ragged last tile
     (6, 15, 64, 128256),      # n_pad 96, two overflow tiles
+    (1, 8, 2048, 40000),      # n_pad 16 with 32 k-slices: early sweep + late sweep on pairs of k-slices
+    (2, 12, 320, 60000),      # odd number of k-slices (5): one slice per ring slot, no paired late sweep
 ]
 
 
@@ -410,6 +412,7 @@ FP8_CASES = [
     ("fused", 4, 16, 128, 40000 + 77),
     ("fused", 1, 25, 512, 128256),
     ("fused", 6, 15, 128, 128256),            # overflow tiles
+    ("fused", 4, 16, 256, 128256),            # 80 padded rows, two k-slices of codes: early sweep + paired late sweep
     ("batched", 8, 16, 128, 128256),          # two row blocks of the FP8 GEMM, the second mostly padding
     ("batched", 3, 50, 256, 5000 + 77),       # ragged last vocabulary block, two k-steps
     ("batched", 64, 16, 128, 20000),          # the serving shape's rows

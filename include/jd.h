@@ -229,6 +229,15 @@ jd_status_t jd_last_launch_info(jd_handle_t h, int* variant, int* kernel_launche
  * fetch W once can approach. Asynchronous on the stream; uses the current device. */
 jd_status_t jd_stream_read_probe(const void* data, size_t bytes, uint32_t* out, void* cuda_stream);
 
+/* Measurement aid (the paper has no counterpart). A library built with -DJD_PHASE_STAMPS
+ * (python -m paper_2501_19309_b200.build --stamps) makes thread 0 of every CTA of the fused kernel
+ * record the GPU's global timer at the phase boundaries of the call; this function copies the
+ * stamps of the most recent fused launch on the current device to the HOST array `out`:
+ * 256 CTAs x 16 slots of nanosecond values (capacity >= 4096 entries), slot meanings as printed by
+ * paper_2501_19309_b200/phase_times.py. Synchronise the stream first. The normal library records
+ * nothing and returns JD_ERR_UNSUPPORTED. */
+jd_status_t jd_debug_phase_stamps(uint64_t* out, int32_t capacity);
+
 /* Test helper: fills out[i] = Philox uniform for (seed, b[i], slot[i], stream[i]), i < n, with
  * the device generator; device pointers. Used to compare the generator bit for bit with an
  * independent host implementation. */

@@ -1,6 +1,9 @@
 """Builds the C-ABI library ``libjd_b200.so`` in-tree with nvcc for sm_100a.
 
-Usage: ``python -m paper_2501_19309_b200.build [--force] [--verbose]``
+Usage: ``python -m paper_2501_19309_b200.build [--force] [--verbose] [--stamps]``
+
+``--stamps`` builds ``libjd_b200_stamps.so`` instead: the same sources with ``-DJD_PHASE_STAMPS``, in which the
+fused kernel records the global timer at its phase boundaries (read with ``phase_times.py``).
 """
 from __future__ import annotations
 
@@ -12,6 +15,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libjd_b200.so")
+LIB_STAMPS = os.path.join(PKG, "libjd_b200_stamps.so")
 SOURCES = ["jd_api.cu", "jd_simt.cu", "jd_fused_sm100.cu", "jd_batched_sm100.cu", "jd_static.cu"]
 HEADERS = ["jd_common.cuh", "jd_kernels.h", "jd_sm100_ptx.cuh"]
 
@@ -31,22 +35,28 @@ def needs_build() -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, stamps: bool = False) -> str:
+    if stamps:
+        return _compile(LIB_STAMPS, verbose, ["-DJD_PHASE_STAMPS"])
     if not force and not needs_build():
         return LIB
+    return _compile(LIB, verbose, [])
+
+
+def _compile(out: str, verbose: bool, defines: list) -> str:
     cmd = [_nvcc(), "-shared", "-Xcompiler", "-fPIC", "-std=c++17", "-O3", "-lineinfo",
            "-gencode", "arch=compute_100a,code=sm_100a",
-           "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+           "-I", os.path.join(ROOT, "include"), "-I", CSRC] + defines
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]
+    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", out]
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or proc.returncode != 0:
         sys.stderr.write(proc.stdout + proc.stderr)
     if proc.returncode != 0:
-        raise RuntimeError("nvcc failed building %s" % LIB)
-    return LIB
+        raise RuntimeError("nvcc failed building %s" % out)
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, stamps="--stamps" in sys.argv))

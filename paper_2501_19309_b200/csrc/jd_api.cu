@@ -565,6 +565,12 @@ jd_status_t jd_selftest_stale_timeout(jd_handle_t h, void* cuda_stream) {
   return JD_OK;   // on purpose not remembered on the host: the device-side rule is what is being tested
 }
 
+jd_status_t jd_debug_phase_stamps(uint64_t* out, int32_t capacity) {
+  if (!out || capacity < kMaxCtas * kPhaseStampSlots) return JD_ERR_INVALID_ARG;
+  static_assert(sizeof(uint64_t) == sizeof(unsigned long long), "stamp type");
+  return read_phase_stamps(reinterpret_cast<unsigned long long*>(out)) ? JD_OK : JD_ERR_UNSUPPORTED;
+}
+
 jd_status_t jd_stream_read_probe(const void* data, size_t bytes, uint32_t* out, void* cuda_stream) {
   if (!data || !out || bytes < 16 || !aligned16(data)) return JD_ERR_INVALID_ARG;
   int dev = 0, sms = 0;

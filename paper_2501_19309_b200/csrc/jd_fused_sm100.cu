@@ -40,6 +40,23 @@
 
 namespace jd {
 
+// Measurement aid, compiled in only with -DJD_PHASE_STAMPS (a library of its own, see build.py): thread 0
+// of every CTA writes the global timer at the phase boundaries of the epilogue, so that a host tool can
+// print where a call's time goes. In the normal build JD_STAMP expands to nothing.
+#ifdef JD_PHASE_STAMPS
+__device__ unsigned long long g_phase_stamps[kMaxCtas * kPhaseStampSlots];
+#define JD_STAMP(n)                                                      \
+  do {                                                                   \
+    if (tid == 0) {                                                      \
+      unsigned long long t_;                                             \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));             \
+      g_phase_stamps[cta * kPhaseStampSlots + (n)] = t_;                 \
+    }                                                                    \
+  } while (0)
+#else
+#define JD_STAMP(n) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int kThreads = 192;
@@ -287,6 +304,10 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   }
   tc_fence_after();
   const uint32_t tmem_base = ms.tmem_base;   // (not meaningful in the producer warp, which does not use it)
+#ifdef JD_PHASE_STAMPS
+  if (tid == 0) g_phase_stamps[cta * kPhaseStampSlots + 13] = g_phase_stamps[cta * kPhaseStampSlots + 11];   // previous launch's end
+#endif
+  JD_STAMP(0);
   if (tid < R) {   // rows whose drafted token this CTA's slice holds (usually none or one)
     const int x = ms.x_row[tid];
     if (x >= t0 * kVocabTile && x < (t0 + T) * kVocabTile) ms.glist[atomicAdd(&ms.glist_n, 1)] = tid;
@@ -549,6 +570,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (lane == 0) ws.judge_logit[bm] = acc;
     }
 
+    JD_STAMP(1);
     // (c)-(e) row statistics, in one or two phases. Phase 1 covers the tiles of the last sweep and
     // starts when the whole accumulation is complete. A CTA that ran an early sweep (T_early > 0)
     // first takes, in phase 0, the statistics of the early tiles while the last sweep still streams,
@@ -569,6 +591,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       epi_sync();
       tc_fence_after();
       ok = ok && (*abort_flag == 0);
+      if (ph == 1) JD_STAMP(2); else JD_STAMP(12);
       const int i_lo = ph == 0 ? 0 : T_early, i_hi = ph == 0 ? T_early : T;
       if constexpr (kSampleOnly) {
         // (h) mass of the sampling weights of each selected row over the phase's tiles.
@@ -726,6 +749,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
       epi_sync();
     }
+    JD_STAMP(3);
     if constexpr (!kSampleOnly) {
     if (ok && cp.logits_debug != nullptr)
       dump_logits<N_PAD>(cp.logits_debug, T, t0, R, V, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0]);
@@ -741,6 +765,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     epi_sync();
     ok = (*abort_flag == 0);
+    JD_STAMP(4);
 
     // (f0) top-K rule: over the parked tiles, count the entries of every draft row that rank above
     // the drafted token (its logit is known grid-wide since barrier 1) and note the lowest token id
@@ -832,6 +857,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
       }
     }
+    JD_STAMP(5);
     __threadfence();
     epi_sync();
 
@@ -844,6 +870,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     epi_sync();
     ok = (*abort_flag == 0);
+    JD_STAMP(6);
     if (ok) {
       if (tid < R) ms.lse[tid] = __ldcg(ws.row_lse + tid);
       if (tid < BM) ms.qlse[tid] = __ldcg(ws.q_lse + tid);
@@ -867,6 +894,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 
     }
 
+    JD_STAMP(7);
     // top-K rule: the next token is the argmax of the selected row; CTA 0 folds the per-CTA maxima
     // and their candidates (larger value first, then lower token id). Nothing is drawn.
     constexpr bool draw = !kTopK;
@@ -952,6 +980,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       ws.mass_r[(size_t)tid * G + cta] = (ms.wd_r[tid][0] + ms.wd_r[tid][1]) + (ms.wd_r[tid][2] + ms.wd_r[tid][3]);
       ws.mass_p[(size_t)tid * G + cta] = (ms.wd_p[tid][0] + ms.wd_p[tid][1]) + (ms.wd_p[tid][2] + ms.wd_p[tid][3]);
     }
+    JD_STAMP(8);
     __threadfence();
     epi_sync();
 
@@ -964,6 +993,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
     epi_sync();
     ok = (*abort_flag == 0);
+    JD_STAMP(9);
 
     // (i) inverse CDF in ascending token id. First, one warp per sequence finds the CTA whose
     // slice contains T = u * total (same arithmetic in every CTA, so every CTA agrees) ...
@@ -1037,6 +1067,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
     }
     epi_sync();
+    JD_STAMP(10);
     // ... then the owning CTA finds the tile from the tile masses and the token inside that tile
     if (ok && draw) {
       for (int b = 0; b < cp.B; ++b) {
@@ -1116,6 +1147,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         if (tid == 0) cp.next_token[b] = token < 0 ? 0 : token;
       }
     }
+    JD_STAMP(11);
     // Every barrier of this launch lies behind CTA 0 now and nothing can report any more: clear the set
     // the previous launch used and publish this launch as done (the next one then takes that set).
     if (!fp.plain_status && cta == 0 && tid == 0 && ok) {
@@ -1164,6 +1196,15 @@ __global__ void timeout_probe_kernel(Workspace ws, unsigned limit) {
 }
 
 }  // namespace
+
+bool read_phase_stamps(unsigned long long* host_out) {
+#ifdef JD_PHASE_STAMPS
+  return cudaMemcpyFromSymbol(host_out, g_phase_stamps, sizeof(unsigned long long) * kMaxCtas * kPhaseStampSlots) == cudaSuccess;
+#else
+  (void)host_out;
+  return false;
+#endif
+}
 
 void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st) {
   timeout_probe_kernel<<<2, 32, 0, st>>>(ws, limit);

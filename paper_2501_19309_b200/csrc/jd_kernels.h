@@ -38,6 +38,13 @@ struct FusedPlan {
 constexpr int kMaxDynamicSmem = 227 * 1024;
 bool fused_configure();
 bool batched_configure();
+// Phase stamps of the fused kernel's last launch (builds with -DJD_PHASE_STAMPS only; false otherwise):
+// kMaxCtas x kPhaseStampSlots global-timer values in ns, slot = 0 start of the epilogue, 1 draft statistics and
+// judge dots done, 12 early sweep complete, 2 stream complete, 3 row statistics done, 4 barrier 1 passed,
+// 5 fold done, 6 barrier 2 passed, 7 decisions done, 8 sampling masses done, 9 barrier 3 passed, 10 owner
+// found, 11 end of the epilogue, 13 the previous launch's slot 11.
+constexpr int kPhaseStampSlots = 16;
+bool read_phase_stamps(unsigned long long* host_out);
 void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st);
 void launch_stale_timeout(const Workspace& ws, cudaStream_t st);
 bool fused_supported(int dtype, int R, int d, int V, int num_sms, FusedPlan* plan);

@@ -14,7 +14,8 @@ import ctypes as C
 import os
 from typing import Optional
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libjd_b200.so")
+# JD_LIBRARY selects another build of the same library (the phase-stamp build of build.py --stamps)
+_LIB_PATH = os.environ.get("JD_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libjd_b200.so")
 _lib = None
 
 JD_OK, JD_ERR_INVALID_ARG, JD_ERR_UNSUPPORTED, JD_ERR_ARCH = 0, 1, 2, 3
@@ -34,7 +35,8 @@ VARIANTS = {"auto": JD_VARIANT_AUTO, "simt": JD_VARIANT_SIMT, "fused": JD_VARIAN
 EXPORTS = ["jd_version", "jd_status_string", "jd_workspace_bytes", "jd_create", "jd_destroy", "jd_set_head",
            "jd_verify", "jd_verify_host", "jd_last_device_status", "jd_last_launch_info", "jd_philox_uniforms",
            "jd_verify_static", "jd_set_head_fp8", "jd_selftest_timeout", "jd_stream_read_probe",
-           "jd_quantize_rows_e4m3", "jd_check_workspace_guards", "jd_selftest_stale_timeout"]
+           "jd_quantize_rows_e4m3", "jd_check_workspace_guards", "jd_selftest_stale_timeout",
+           "jd_debug_phase_stamps"]
 
 
 class jd_config_t(C.Structure):
@@ -92,6 +94,7 @@ def load():
     lib.jd_quantize_rows_e4m3.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.jd_check_workspace_guards.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
     lib.jd_selftest_stale_timeout.argtypes = [C.c_void_p, C.c_void_p]
+    lib.jd_debug_phase_stamps.argtypes = [C.c_void_p, C.c_int32]
     for name in EXPORTS:
         if name not in ("jd_version", "jd_status_string", "jd_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -143,6 +146,11 @@ def jd_verify_host(h, args: jd_verify_args_t, stream_ptr: int = 0) -> int:
 
 def jd_selftest_timeout(h, spin_limit: int, stream_ptr: int = 0) -> int:
     return load().jd_selftest_timeout(h, C.c_uint32(spin_limit), C.c_void_p(stream_ptr))
+
+
+def jd_debug_phase_stamps(out_ptr: int, capacity: int) -> int:
+    """Copies the fused kernel's phase stamps into a host array of uint64 (stamps build only); see jd.h."""
+    return load().jd_debug_phase_stamps(C.c_void_p(out_ptr), C.c_int32(capacity))
 
 
 def jd_selftest_stale_timeout(h, stream_ptr: int = 0) -> int:

@@ -36,6 +36,11 @@ def test_calls_that_need_no_device():
     assert 1 << 20 < n < 1 << 30
     bad = jd.jd_config_t(0, 16, 8192, 128256, jd.JD_DTYPE_BF16, 0)
     assert jd.jd_workspace_bytes(bad) == 0
+    # the normal build records no phase stamps and says so; bad arguments are refused first
+    buf = (ctypes.c_uint64 * 4096)()
+    assert jd.jd_debug_phase_stamps(ctypes.addressof(buf), 4096) == jd.JD_ERR_UNSUPPORTED
+    assert jd.jd_debug_phase_stamps(ctypes.addressof(buf), 100) == jd.JD_ERR_INVALID_ARG
+    assert jd.jd_debug_phase_stamps(0, 4096) == jd.JD_ERR_INVALID_ARG
 
 
 def test_struct_layout_matches_header_order():

@@ -68,7 +68,7 @@ typedef enum { JD_RESAMPLE_RESIDUAL = 0, JD_RESAMPLE_TARGET_P = 1 } jd_resample_
  * SAMPLING: the stochastic test of Eq. 4 with the residual / bonus draw described above.
  * TOPK:     deterministic verification: the candidate passes iff it is among the top_k highest-valued
  *           entries of p_j (Sec. 5.1 "Training-free baseline"); top_k = 1 is greedy verification
- *           (acceptance "under greedy decoding", Sec. 3.2), top_k = V accepts everything. The next
+ *           (acceptance against a greedily decoded target, Sec. 3.2), top_k = V accepts everything. The next
  *           token is the target's greedy token argmax p_a, at a rejection and after a full block.
  *           Equal logits rank by token id (lower id first). No uniform is drawn; the draft logits
  *           only feed the q_draft output. */

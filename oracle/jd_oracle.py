@@ -18,13 +18,13 @@ Sec. 4.1 "Inference"; 0-indexed here, the paper is 1-indexed):
       s[j]       = sigmoid(w . H[b, j+1] + b0)   judge score of x_j's own embedding
       z_judge[j] = s[j] > tau                    (Sec. 4.1 "Inference")
       z[j]       = z_std[j] or z_judge[j]        (or one of them, by mode)
-  a = index of the first j with z[j] == 0, else M   ("if all previous tokens are accepted")
+  a = index of the first j with z[j] == 0, else M   (a token counts only while all before it were accepted)
   next token: from the residual max(0, p_a - q_a), normalised, when a < M;
               from p_M after a fully accepted block; inverse CDF in ascending
               token id with one uniform.
 
-Deterministic variants of the standard test (Sec. 3.2 speaks of acceptance "under greedy
-decoding"; Sec. 5.1 "Training-free baseline" defines top-K verification): with rule="topk" the
+Deterministic variants of the standard test (Sec. 3.2 measures acceptance with a greedily
+decoded target; Sec. 5.1 "Training-free baseline" defines top-K verification): with rule="topk" the
 candidate x_j passes the standard test iff it is among the K highest-valued entries of p_j
 (K = 1 is greedy verification, K = V accepts everything), and the next token is the target's
 greedy token argmax p_a, at a rejection as well as after a fully accepted block. No uniform is
@@ -32,7 +32,7 @@ drawn and the draft distribution plays no role. Equal logits are ordered by toke
 ranks higher), so "among the K highest" and "argmax" are unique.
 
 Final RMS normalisation (Sec. 4.1 "Model design and training": the judge reads the last embedding
-"before the RMS normalization and the LM head"): with rms_eps given, the LM head sees
+ahead of the model's final RMS norm and LM head): with rms_eps given, the LM head sees
 H[b,j] / sqrt(mean_k H[b,j,k]^2 + rms_eps) while the judge still reads H[b,j+1] itself. The
 normalisation gain is taken as folded into W beforehand.
 
@@ -48,8 +48,8 @@ Readings taken where the paper is silent (all restated in the design notes):
   * the judge for draft token j reads row j+1 of H, the embedding produced by
     feeding that token (Sec. 4.1 speaks of the embedding of the current token);
   * the token at the first rejection comes from the residual distribution, the
-    form that keeps standard speculative sampling lossless; the paper's literal
-    "sample from p_i" is available as resample="target_p";
+    form that keeps standard speculative sampling lossless; the paper's wording taken
+    literally (draw from p_i itself) is available as resample="target_p";
   * Eq. 4 is evaluated division-free, u*q < p, which equals u < min(1, p/q)
     for u in [0, 1); q(x) = 0 accepts iff p(x) > 0;
   * the judge comparison is strict; tau = 1 never accepts, so the OR mode

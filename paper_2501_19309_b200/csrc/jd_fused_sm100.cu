@@ -332,7 +332,8 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
   // The other sweeps, too, move two k-slices per ring slot whenever d allows it (kk = 2): one wait and one
   // commit then serve eight MMAs of a tile instead of four, which keeps the producer and MMA threads'
   // per-tile work safely below the time HBM needs for the tile's bytes.
-  const int kk = (fp.num_kb & 1) == 0 ? 2 : 1;
+  // (not with rings too short for two slots each: 81 to 96 rows at the full vocabulary leave three W slices)
+  const int kk = ((fp.num_kb & 1) == 0 && fp.stages >= 4 && fp.h_stages >= 4) ? 2 : 1;
   const int w_slots = fp.stages / kk, h_slots = fp.h_stages / kk;   // ring depths in slots of kk slices
 
   if (warp == 4 && lane == 0) {
@@ -627,9 +628,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
               float d0[16], d1[16], v0[16], v1[16];
 #pragma unroll
               for (int k = 0; k < 16; ++k) {
-                const int kk = min(k, cp.B - 1 - min(c0, cp.B - 1));   // stay inside the buffer in a ragged last chunk
-                d0[k] = __ldg(base0 + kk * kVocabTile);
-                d1[k] = __ldg(base1 + kk * kVocabTile);
+                const int ks = min(k, cp.B - 1 - min(c0, cp.B - 1));   // stay inside the buffer in a ragged last chunk
+                d0[k] = __ldg(base0 + ks * kVocabTile);
+                d1[k] = __ldg(base1 + ks * kVocabTile);
               }
               load_chunk2<N_PAD>(i0, i_hi, c0, n_ovf, ts, tmem_lane_base, ovf, tid, ms.scale, &ms.swt[0][0], v0, v1);
 #pragma unroll

@@ -27,6 +27,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import re
 import statistics
 import subprocess
 import sys
@@ -211,10 +212,36 @@ def roofline_of(wl: I.Workload, peaks: dict, kernel_ms: float, sustained: bool, 
             "kernel_ms": kernel_ms}
 
 
-def oracle_step(inp: I.Inputs, seed: int, sequences):
+RMS_EPS = 1e-5          # the epsilon of the RMSNorm option where a workload token asks for it
+NO_OPTIONS = {"rule": "sampling", "top_k": 1, "rms_eps": None}
+
+
+def parse_workload_token(tok: str):
+    """'<id>[f][g|k][n]': workload id, then f = FP8 E4M3 head, g = greedy rule (top-K with K = 1),
+    k = top-5 rule, n = final RMSNorm ahead of the LM head. Returns (workload or None, options)."""
+    m = re.fullmatch(r"(\d+)(f?)([gk]?)(n?)", tok)
+    if not m or int(m.group(1)) not in I.CONFIGS:
+        return None, None
+    wl = I.CONFIGS[int(m.group(1))]
+    name = wl.name + ("-fp8" if m.group(2) else "")
+    opts = dict(NO_OPTIONS)
+    if m.group(3):
+        opts.update(rule="topk", top_k=1 if m.group(3) == "g" else 5)
+        name += "-greedy" if m.group(3) == "g" else "-top5"
+    if m.group(4):
+        opts["rms_eps"] = RMS_EPS
+        name += "-rmsnorm"
+    if name != wl.name:
+        wl = wl.scaled(name, dtype="fp8" if m.group(2) else wl.dtype)
+    return wl, opts
+
+
+def oracle_step(inp: I.Inputs, seed: int, sequences, opts=None):
     from oracle import jd_oracle as O
+    o = opts or NO_OPTIONS
     return O.jd_oracle_verify(inp.W, inp.w_judge, inp.b_judge, inp.H, inp.draft_tokens, inp.draft_logits,
-                              inp.tau, seed, "judge_or_standard", sequences=sequences, w_scale=inp.w_scale)
+                              inp.tau, seed, "judge_or_standard", sequences=sequences, w_scale=inp.w_scale,
+                              rule=o["rule"], top_k=o["top_k"], rms_eps=o["rms_eps"])
 
 
 def cpu_threads() -> int:
@@ -249,7 +276,7 @@ def time_oracle(inp: I.Inputs, steps: int, budget_s: float = 25.0, extra_warmup:
             "seconds": dt, "first": first}
 
 
-def parity_of(wl: I.Workload, got: dict, ref) -> dict:
+def parity_of(wl: I.Workload, got: dict, ref, rule: str = "sampling") -> dict:
     """Device outputs of verify seed 0 against the checker's result for the same inputs, under the
     rules of the parity tests (tests/jd_testlib.py: tolerances, margin exemptions, CDF intervals)."""
     tests_dir = os.path.join(ROOT, "tests")
@@ -258,7 +285,7 @@ def parity_of(wl: I.Workload, got: dict, ref) -> dict:
     import jd_testlib as T
     rep = T.Report()
     try:
-        T.compare(got, ref, "judge_or_standard", wl.M, rep)
+        T.compare(got, ref, "judge_or_standard", wl.M, rep, rule=rule)
         ok, why = True, None
     except AssertionError as e:
         ok, why = False, str(e)[:200]
@@ -308,8 +335,9 @@ def log(msg: str) -> None:
     sys.stderr.flush()
 
 
-def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
+def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks, opts=None):
     """Times K device-resident calls and K_e2e host-buffer calls of one workload on this rank."""
+    o = dict(opts or NO_OPTIONS)
     log("%s: drawing inputs" % wl.name)
     inp = I.make_inputs(wl, data_seed)
     log("%s: inputs drawn" % wl.name)
@@ -323,7 +351,7 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     ver = jd.Verifier(wl.B, wl.M, wl.d, wl.V, "fp8" if fp8 else "bf16", device.index)
     ver.set_head(W, w, inp.b_judge, w_scale=w_scale)
     out = ver.alloc_outputs(wl.B, wl.M)
-    a_args = [ver.make_args(H, x, dl, inp.tau, s, "judge_or_standard", out=out)[0] for s in range(8)]
+    a_args = [ver.make_args(H, x, dl, inp.tau, s, "judge_or_standard", out=out, **o)[0] for s in range(8)]
     stream = torch.cuda.current_stream(device)
 
     def step(i):
@@ -414,7 +442,7 @@ def measure_workload(wl, args, torch, jd, device, data_seed, sample_clocks):
     hx = torch.from_numpy(inp.draft_tokens).pin_memory()
     hdl = torch.from_numpy(inp.draft_logits).pin_memory()
     hout = ver.alloc_outputs(wl.B, wl.M, host=True)
-    h_args = [ver.make_args(hH, hx, hdl, inp.tau, s, "judge_or_standard", out=hout, host=True)[0] for s in range(8)]
+    h_args = [ver.make_args(hH, hx, hdl, inp.tau, s, "judge_or_standard", out=hout, host=True, **o)[0] for s in range(8)]
     Ke = max(3, min(K, args.e2e_steps))
     for i in range(3):
         jd.jd_verify_host(ver.h, h_args[i % 8], stream.cuda_stream)
@@ -450,7 +478,7 @@ def main() -> None:
     ap.add_argument("--config", type=int, default=3, help="workload id of the headline line (1..4); default: the "
                     "405B-shaped head, the largest single-GPU configuration")
     ap.add_argument("--others", default="2,1,4,3f,4f", help="comma list of further workloads summarised in the same "
-                    "line; a trailing f = the same shape with an FP8 E4M3 head")
+                    "line: an id, then f = FP8 E4M3 head, g / k = greedy / top-5 rule, n = RMSNorm ahead of the head")
     ap.add_argument("--record-traffic", nargs="+", metavar="WORKLOAD=CSV[,CSV]", help="rewrite profiles/ncu_traffic.json "
                     "from ncu raw-page CSV exports and exit")
     ap.add_argument("--fp8", action="store_true", help="headline workload with an FP8 E4M3 head")
@@ -498,19 +526,15 @@ def main() -> None:
         small = argparse.Namespace(**vars(args))
         small.dist = False
         for tok in [c.strip() for c in args.others.split(",") if c.strip()]:
-            as_fp8 = tok.endswith("f")
-            cid = int(tok.rstrip("f"))
-            if (cid == args.config and not as_fp8) or cid not in I.CONFIGS:
+            owl, oopts = parse_workload_token(tok)
+            if owl is None or owl.name == wl.name:
                 continue
-            owl = I.CONFIGS[cid]
-            if as_fp8:
-                owl = owl.scaled(owl.name + "-fp8", dtype="fp8")
             small.steps = max(50, min(args.steps, 300))
             small.e2e_steps = 10
-            r = measure_workload(owl, small, torch, jd, device, data_seed=0, sample_clocks=True)
+            r = measure_workload(owl, small, torch, jd, device, data_seed=0, sample_clocks=True, opts=oopts)
             oparity = None
             if not args.no_cpu_baseline:      # the checker on the first sequence of this workload
-                oparity = parity_of(owl, r["out0"], oracle_step(r["inp"], 0, [0]))
+                oparity = parity_of(owl, r["out0"], oracle_step(r["inp"], 0, [0], oopts), rule=oopts["rule"])
             e2e_note = None
             if owl.B * owl.M * owl.V * 4 > 100e6:
                 e2e_note = ("%.0f MB of fp32 draft logits cross PCIe per host-buffer call" % (owl.B * owl.M * owl.V * 4 / 1e6))
@@ -518,7 +542,8 @@ def main() -> None:
                 "B": owl.B, "M": owl.M, "d": owl.d, "V": owl.V, "ms_per_step": r["mean_ms"],
                 "median_ms": r["median_ms"], "value": owl.B * owl.M / (r["mean_ms"] * 1e-3), "unit": UNIT,
                 "variant": VARIANT_NAMES.get(r["variant"], "?"), "kernel_launches_per_step": r["launches"],
-                "steps": small.steps, "mean_accept_len": r["mean_accept"], "best_ms": r["min_ms"],
+                "rule": oopts["rule"] if oopts["rule"] == "sampling" else "top-%d" % oopts["top_k"],
+                "norm": "rms" if oopts["rms_eps"] else "none", "steps": small.steps, "mean_accept_len": r["mean_accept"], "best_ms": r["min_ms"],
                 "clocks": r["clocks"],
                 "graph_replay_ms_per_step": r["graph_ms"],
                 "emitted_tokens_per_s": r["emitted_per_call"] / (r["mean_ms"] * 1e-3),

@@ -163,6 +163,7 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws, size_t* guard_off 
   w.cnt = (int*)take(maxR * 4);
   w.argidx = (int*)take(maxR * 4);
   w.part_idx = (int*)take(maxR * np * 4);
+  w.cand_ref = (float*)take(maxR * 4);
   w.status = (unsigned*)take(512);   // status word and, 256 bytes on, the barrier counters: one memset per call
   w.barrier = w.status ? w.status + 64 : nullptr;
   char* flag = take(256);   // word 0: arrival flag of a host-buffer call's draft logits; outside the per-call memset
@@ -420,7 +421,7 @@ jd_status_t jd_verify(jd_handle_t h, const jd_verify_args_t* a, void* cuda_strea
       return JD_ERR_CUDA;
     cudaError_t err = cudaSuccess;
     const int n = run_batched(cp, h->ws, h->tm_w256, h->tm_w, tm_h, tm_hsel, tm_hsel_tail, a->H, h->w_judge, h->num_sms,
-                              st, h->side, &err, fp8 ? h->w_scale : nullptr);
+                              st, h->side, &err, fp8 ? h->w_scale : nullptr, h->W);
     if (n < 0) return JD_ERR_CUDA;
     launches += n;
   } else {

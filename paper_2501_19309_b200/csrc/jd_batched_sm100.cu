@@ -6,6 +6,10 @@
 //   tensor memory: the epilogue warps turn it into one (max, sum exp) pair per row and pick out
 //   the drafted token's logit, while the next tile's MMAs fill the other half of tensor memory.
 // Then the shared decision kernel folds the per-tile pairs, runs both tests and the prefix rule.
+// With the top-K / greedy rule the same pass also counts, per row, the entries that rank above the
+//   drafted token (against that token's logit, computed ahead of the pass by a small CUDA-core
+//   kernel) and keeps the argmax of every tile: the call is then complete after the fold, and
+//   W is streamed once.
 // Pass 2: the selected row of every sequence (B rows) is gathered and handed to the fused
 //   kernel in its sample-only mode, which recomputes those B rows of logits with W streamed
 //   once more and draws the next tokens.
@@ -57,11 +61,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 //       codes per instruction, 128 per k-step); the epilogue applies the scale of the vocabulary row
 //       and of the H row to every accumulator. A template parameter, so that the MMA loop of one
 //       instantiation names one instruction kind only.
-// kCount == false: softmax statistics + gather (first pass).
-// kCount == true : top-K rule, after the fold: the same GEMM again (bit-identical logits), the
-//                  epilogue counts the entries that rank above the drafted token and records the
-//                  lowest token id equal to the folded row maximum.
-template <bool kCount, bool kFp8>
+// kTopK == false: softmax statistics + gather of the drafted token's logit.
+// kTopK == true : the same, and for the top-K / greedy rule the epilogue also counts the entries of the
+//                 row that rank above the drafted token (its logit is in ws.cand_ref before the kernel
+//                 starts; the token's own column is left out of the count, ties rank by token id) and
+//                 records the lowest token id that attains the tile's maximum.
+template <bool kTopK, bool kFp8>
 __global__ void __launch_bounds__(kBThreads, 1)
 gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmH, CallParams cp,
                   Workspace ws, int R, int np, const float* __restrict__ w_scale) {
@@ -176,14 +181,11 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       tc_fence_after();
       float m = -INFINITY, s = 0.f, g = 0.f;
       bool have_g = false;
-      int above = 0, cand = 0x7F7F7F7F;
-      float g_ref = 0.f, rmax = 0.f;
+      int above = 0, arg = 0x7F7F7F7F;
+      float g_ref = 0.f;
       float sc = (cp.norm == JD_NORM_RMS && row < R) ? ws.row_scale[row] : 1.f;
       if (kFp8 && row < R) sc *= ws.h_scale[row];
-      if (kCount && row < R) {
-        rmax = ws.row_max[row];
-        if (x >= 0) g_ref = ws.gath[row];
-      }
+      if (kTopK && x >= 0) g_ref = ws.cand_ref[row];
 #pragma unroll 1
       for (int c0 = 0; c0 < kTileN; c0 += 32) {
         float v[32];
@@ -196,7 +198,7 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
           for (int k = 0; k < 32; ++k) v[k] *= sc;
         }
         const int nvalid = cp.V - (v0 + c0);   // columns of this chunk that exist (>= 32 except at the tail)
-        if (!kCount && cp.logits_debug != nullptr && row < R) {   // test-only copy of the logits
+        if (cp.logits_debug != nullptr && row < R) {   // test-only copy of the logits
           float* o = cp.logits_debug + (size_t)row * cp.V + v0 + c0;
 #pragma unroll
           for (int k = 0; k < 32; ++k) if (k < nvalid) o[k] = v[k];
@@ -205,18 +207,22 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 #pragma unroll
           for (int k = 0; k < 32; ++k) if (k >= nvalid) v[k] = -INFINITY;
         }
-        if (kCount) {
-#pragma unroll
-          for (int k = 0; k < 32; ++k) {
-            const int col = v0 + c0 + k;
-            if (x >= 0 && (v[k] > g_ref || (v[k] == g_ref && col < x))) ++above;
-            if (v[k] == rmax) cand = min(cand, col);
-          }
-          continue;
-        }
         float cm = v[0];
 #pragma unroll
         for (int k = 1; k < 32; ++k) cm = fmaxf(cm, v[k]);
+        if (kTopK) {
+          if (x >= 0) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+              const int col = v0 + c0 + k;
+              if (col != x && (v[k] > g_ref || (v[k] == g_ref && col < x))) ++above;
+            }
+          }
+          if (cm > m) {   // a new maximum of the tile: its first column in this chunk
+#pragma unroll
+            for (int k = 31; k >= 0; --k) if (v[k] == cm) arg = v0 + c0 + k;
+          }
+        }
         const float mn = fmaxf(m, cm);
         if (mn > -INFINITY) {
           const float off = mn * kLog2e;
@@ -236,13 +242,12 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       epi_sync();
       if (tid == 0) mbar_arrive(smem_u32(&ms.tmem_empty[buf]));
       if (row < R) {
-        if (kCount) {
+        ws.part_max[(size_t)row * np + vb] = m;
+        ws.part_sum[(size_t)row * np + vb] = s;
+        if (have_g) ws.gath[row] = g;
+        if (kTopK) {
           if (above) atomicAdd(ws.cnt + row, above);
-          if (cand != 0x7F7F7F7F) atomicMin(ws.argidx + row, cand);
-        } else {
-          ws.part_max[(size_t)row * np + vb] = m;
-          ws.part_sum[(size_t)row * np + vb] = s;
-          if (have_g) ws.gath[row] = g;
+          ws.part_idx[(size_t)row * np + vb] = arg;
         }
       }
     }
@@ -257,6 +262,50 @@ gemm_stats_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   if (warp == 5) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// Top-K / greedy rule: the logit of every drafted token, L[row, x] = H[row] . W[x] with the scales the
+// GEMM's epilogue applies, on CUDA cores ahead of the GEMM pass (one CTA per row, 2 x d elements read).
+// The pass ranks the other entries of the row against this value; it differs from the tensor cores'
+// own L[row, x] by float32 summation order only, and that column is left out of the count.
+template <bool kFp8>
+__global__ void __launch_bounds__(128) candidate_logit_kernel(CallParams cp, Workspace ws, const uint8_t* __restrict__ W,
+                                                              const uint8_t* __restrict__ H,
+                                                              const float* __restrict__ w_scale) {
+  __shared__ float part[4];
+  const int row = blockIdx.x, tid = threadIdx.x;
+  const int b = row / (cp.M + 1), j = row % (cp.M + 1);
+  if (j >= cp.M) return;
+  const int x = min(max(cp.draft_tokens[b * cp.M + j], 0), cp.V - 1);   // the GEMM pass reports a bad token
+  const int row_bytes = kFp8 ? cp.d : cp.d * 2;
+  const uint4* wr = reinterpret_cast<const uint4*>(W + (size_t)x * row_bytes);
+  const uint4* hr = reinterpret_cast<const uint4*>(H + (size_t)row * row_bytes);
+  float acc = 0.f;
+  for (int k = tid; k < row_bytes / 16; k += 128) {
+    const uint4 a = __ldg(wr + k), h = __ldg(hr + k);
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, hw[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (kFp8) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          acc = fmaf(to_float(e4m3_t{(uint8_t)(aw[q] >> (8 * e))}), to_float(e4m3_t{(uint8_t)(hw[q] >> (8 * e))}), acc);
+      } else {
+        acc = fmaf(__uint_as_float(aw[q] << 16), __uint_as_float(hw[q] << 16), acc);
+        acc = fmaf(__uint_as_float(aw[q] & 0xFFFF0000u), __uint_as_float(hw[q] & 0xFFFF0000u), acc);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((tid & 31) == 0) part[tid >> 5] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    float v = (part[0] + part[1]) + (part[2] + part[3]);
+    float sc = cp.norm == JD_NORM_RMS ? ws.row_scale[row] : 1.f;
+    if (kFp8) { sc *= ws.h_scale[row]; v *= __ldg(w_scale + x); }
+    ws.cand_ref[row] = v * sc;
   }
 }
 
@@ -312,24 +361,29 @@ bool batched_supported(int dtype, int B, int d, int V, int num_sms) {
 int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
                 const CUtensorMap& tmH, const CUtensorMap& tmHsel, const CUtensorMap& tmHselTail, const void* H,
                 const void* w_judge, int num_sms, cudaStream_t st, const SideStream& side, cudaError_t* err,
-                const float* w_scale_fp8) {
+                const float* w_scale_fp8, const void* W) {
   const bool fp8 = w_scale_fp8 != nullptr;
   const int dtype = fp8 ? JD_DTYPE_FP8_E4M3 : JD_DTYPE_BF16;
   const int R = cp.B * (cp.M + 1);
   const int np = (cp.V + kTileN - 1) / kTileN;
   const size_t smem = 1024 + kBMisc + (size_t)kBStages * (kAStage + kBStage);
-  auto gemm = [&](bool count) {
-    auto kern = fp8 ? (count ? gemm_stats_kernel<true, true> : gemm_stats_kernel<false, true>)
-                    : (count ? gemm_stats_kernel<true, false> : gemm_stats_kernel<false, false>);
+  const bool topk = cp.rule == JD_RULE_TOPK;
+  auto gemm = [&]() {
+    auto kern = fp8 ? (topk ? gemm_stats_kernel<true, true> : gemm_stats_kernel<false, true>)
+                    : (topk ? gemm_stats_kernel<true, false> : gemm_stats_kernel<false, false>);
     kern<<<grid_of(R, np, num_sms), kBThreads, smem, st>>>(tmW256, tmH, cp, ws, R, np, w_scale_fp8);
     return true;
   };
+  if (topk) {   // the drafted tokens' logits, which the pass ranks the rows against
+    if (fp8) candidate_logit_kernel<true><<<R, 128, 0, st>>>(cp, ws, (const uint8_t*)W, ws.h8, w_scale_fp8);
+    else candidate_logit_kernel<false><<<R, 128, 0, st>>>(cp, ws, (const uint8_t*)W, (const uint8_t*)H, nullptr);
+  }
   int nq;
   if (side.stream) {
     // The draft statistics (HBM-bound) and the judge dots do not depend on the GEMM (tensor-bound):
     // they run on the handle's side stream next to it and join before the decision.
     if ((*err = cudaEventRecord(side.fork, st)) != cudaSuccess) return -1;
-    if (!gemm(false)) return -1;
+    if (!gemm()) return -1;
     if ((*err = cudaStreamWaitEvent(side.stream, side.fork, 0)) != cudaSuccess) return -1;
     nq = launch_q_stats(cp, ws, side.stream);
     launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, side.stream);
@@ -338,11 +392,10 @@ int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tm
   } else {
     nq = launch_q_stats(cp, ws, st);
     launch_judge(cp, ws, H, w_judge, JD_DTYPE_BF16, st);
-    if (!gemm(false)) return -1;
+    if (!gemm()) return -1;
   }
-  launch_fold(cp, ws, np, nq, st);
-  if (cp.rule == JD_RULE_TOPK) {   // second GEMM pass for ranks and argmax; no token draw
-    if (!gemm(true)) return -1;
+  launch_fold(cp, ws, np, nq, st, /*fold_arg=*/topk);
+  if (topk) {   // ranks and argmax came out of the same pass; the decision writes the token, nothing is drawn
     launch_decide(cp, ws, st);
     return 6;
   }

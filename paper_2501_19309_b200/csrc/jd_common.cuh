@@ -44,7 +44,9 @@ struct Workspace {
   float* row_scale;    // [maxR] 1 / sqrt(mean square + eps) of every row of H (JD_NORM_RMS)
   int* cnt;            // [maxR] top-K rule: entries of the row that rank above the drafted token
   int* argidx;         // [maxR] top-K rule: lowest token id that attains the row maximum
-  int* part_idx;       // [maxR][np] top-K rule, fused variant: per-CTA argmax candidates
+  int* part_idx;       // [maxR][np] top-K rule: per-CTA argmax candidates (fused variant); lowest token id
+                       //            that attains the tile's maximum, per vocabulary tile (batched variant)
+  float* cand_ref;     // [maxR] top-K rule, batched variant: L[row, x_j] computed ahead of the GEMM pass
   __nv_bfloat16* h_sel;  // [maxB][d] selected rows of H gathered for the batched variant's second pass
   unsigned* status;    // [1] device status word: jd_status_t of the first device-side problem in bits 0-7; bits 8-31 a
                        //     call tag when the fused kernel wrote it (see kCallCounter), 0 when another kernel did

@@ -14,7 +14,8 @@ int launch_q_stats(const CallParams& cp, const Workspace& ws, cudaStream_t st); 
 void launch_judge(const CallParams& cp, const Workspace& ws, const void* H, const void* w, int dtype, cudaStream_t st);
 void launch_quantize_rows(const CallParams& cp, const Workspace& ws, const void* H_bf16, cudaStream_t st);
 void launch_row_scale(const CallParams& cp, const Workspace& ws, const void* H, int dtype, cudaStream_t st);
-void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st);
+// fold_arg: also folds the per-tile argmax candidates in ws.part_idx into ws.argidx (batched variant, top-K rule)
+void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st, bool fold_arg = false);
 void launch_decide(const CallParams& cp, const Workspace& ws, cudaStream_t st);
 void launch_locate(const CallParams& cp, const Workspace& ws, int np, cudaStream_t st);
 void launch_stream_read(const void* p, size_t bytes, uint32_t* out, int num_sms, cudaStream_t st);
@@ -78,6 +79,6 @@ bool batched_supported(int dtype, int B, int d, int V, int num_sms);
 int run_batched(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW256, const CUtensorMap& tmW128,
                 const CUtensorMap& tmH, const CUtensorMap& tmHsel, const CUtensorMap& tmHselTail, const void* H,
                 const void* w_judge, int num_sms, cudaStream_t st, const SideStream& side, cudaError_t* err,
-                const float* w_scale_fp8 = nullptr);
+                const float* w_scale_fp8 = nullptr, const void* W = nullptr);
 
 }  // namespace jd

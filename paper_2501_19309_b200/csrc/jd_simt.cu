@@ -358,7 +358,7 @@ __global__ void __launch_bounds__(256) judge_dot_kernel(CallParams cp, Workspace
 // its share of the row's partials (eight at a time, all loads first), the warp takes the
 // maximum, then the rescaled sum; fixed order, so results repeat bit for bit.
 // -----------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) fold_stats_kernel(CallParams cp, Workspace ws, int np, int nq) {
+__global__ void __launch_bounds__(256) fold_stats_kernel(CallParams cp, Workspace ws, int np, int nq, int fold_arg) {
   const int lane = threadIdx.x & 31;
   const int R = cp.B * (cp.M + 1), BM = cp.B * cp.M;
   const int it = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -377,6 +377,13 @@ __global__ void __launch_bounds__(256) fold_stats_kernel(CallParams cp, Workspac
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (fold_arg && is_p) {   // the lowest tile that attains the row maximum holds the lowest such token id
+    int first = 0x7FFFFFFF;
+    for (int i = lane; i < n; i += 32) if (pm[i] == m) first = min(first, i);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) first = min(first, __shfl_xor_sync(0xffffffffu, first, o));
+    if (lane == 0 && first < n) ws.argidx[it] = ws.part_idx[(size_t)it * np + first];
+  }
   float s = 0.f;
   for (int i0 = 0; i0 < n; i0 += 256) {
     float vm[8], vs[8];
@@ -530,9 +537,9 @@ void launch_row_scale(const CallParams& cp, const Workspace& ws, const void* H, 
   else row_scale_kernel<float><<<R, 256, 0, st>>>(cp, ws, (const float*)H);
 }
 
-void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st) {
+void launch_fold(const CallParams& cp, const Workspace& ws, int np, int nq, cudaStream_t st, bool fold_arg) {
   const int items = cp.B * (2 * cp.M + 1);
-  fold_stats_kernel<<<(items + 7) / 8, 256, 0, st>>>(cp, ws, np, nq);
+  fold_stats_kernel<<<(items + 7) / 8, 256, 0, st>>>(cp, ws, np, nq, fold_arg ? 1 : 0);
 }
 
 void launch_decide(const CallParams& cp, const Workspace& ws, cudaStream_t st) {

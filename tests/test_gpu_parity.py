@@ -317,6 +317,18 @@ def test_batched_matches_simt_on_every_sequence(B, M):
         assert np.mean(a["next_token"] == b["next_token"]) > 0.9      # CDF-edge cases may differ by a token
         assert np.allclose(a["row_lse"], b["row_lse"], rtol=0, atol=1e-4)
         assert np.allclose(a["p_draft"], b["p_draft"], rtol=1e-4)
+    # greedy / top-K rule: the batched variant ranks each row in its one GEMM pass against a logit
+    # computed ahead of it; the CUDA-core variant ranks against its own logits in a second pass
+    for k in (1, 3, 50):
+        a = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "judge_or_standard", variant="batched",
+                                  rule="topk", top_k=k))
+        b = T.to_numpy(ver.verify(dev["H"], dev["x"], dev["dl"], 0.5, 0, "judge_or_standard", variant="simt",
+                                  rule="topk", top_k=k))
+        assert ver.device_status() == 0
+        assert np.mean(a["masks"] == b["masks"]) > 0.995              # a near tie at the K-th rank may differ
+        same = a["accept_len"] == b["accept_len"]
+        assert same.mean() > 0.97
+        assert np.array_equal(a["next_token"][same], b["next_token"][same])   # argmax of the same row
     ver.close()
 
 
@@ -330,6 +342,7 @@ TOPK_CASES = [
     ("fused", 6, 15, 64, 40000 + 77, [1, 10]),        # overflow tiles + ragged last tile
     ("batched", 8, 16, 128, 128256, [1, 4]),
     ("batched", 3, 50, 128, 5000 + 77, [1, 100, 5077]),
+    ("batched", 20, 12, 192, 33000 + 5, [1, 2]),      # three row blocks, three k-steps, ragged vocabulary
 ]
 
 

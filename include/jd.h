@@ -70,8 +70,10 @@ typedef enum { JD_RESAMPLE_RESIDUAL = 0, JD_RESAMPLE_TARGET_P = 1 } jd_resample_
  *           entries of p_j (Sec. 5.1 "Training-free baseline"); top_k = 1 is greedy verification
  *           (acceptance against a greedily decoded target, Sec. 3.2), top_k = V accepts everything. The next
  *           token is the target's greedy token argmax p_a, at a rejection and after a full block.
- *           Equal logits rank by token id (lower id first). No uniform is drawn; the draft logits
- *           only feed the q_draft output. */
+ *           Equal logits rank by token id (lower id first); the batched variant compares the row against
+ *           a float32 dot product for the candidate, so there an entry equal to the candidate's logit to
+ *           within float32 summation order may rank on either side of it. No uniform is drawn; the
+ *           draft logits only feed the q_draft output. */
 typedef enum { JD_RULE_SAMPLING = 0, JD_RULE_TOPK = 1 } jd_rule_t;
 
 /* Normalisation applied to the rows of H in front of the LM head. The paper's judge takes the last

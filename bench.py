@@ -253,21 +253,21 @@ def cpu_threads() -> int:
         return os.cpu_count() or 1
 
 
-def time_oracle(inp: I.Inputs, steps: int, budget_s: float = 25.0, extra_warmup: int = 0) -> dict:
+def time_oracle(inp: I.Inputs, steps: int, budget_s: float = 25.0, extra_warmup: int = 0, opts=None) -> dict:
     """The checker as it stands on a bounded sample: whole sequences b = 0, 1, ... of the workload.
     Step s uses verify seed s; "first" is the result of step 0 (kept for the parity check)."""
     wl = inp.wl
     t0 = time.perf_counter()
-    oracle_step(inp, 0, [0])
+    oracle_step(inp, 0, [0], opts)
     one = time.perf_counter() - t0
     for _ in range(extra_warmup):          # untimed, on top of the sizing call above
-        oracle_step(inp, 0, [0])
+        oracle_step(inp, 0, [0], opts)
     nseq = int(max(1, min(wl.B, budget_s / max(one, 1e-3) / max(steps, 1))))
     seqs = list(range(nseq))
     first = None
     t0 = time.perf_counter()
     for s in range(steps):
-        r = oracle_step(inp, s, seqs)
+        r = oracle_step(inp, s, seqs, opts)
         first = first or r
     dt = time.perf_counter() - t0
     return {"value": nseq * wl.M * steps / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
@@ -297,15 +297,18 @@ def parity_of(wl: I.Workload, got: dict, ref, rule: str = "sampling") -> dict:
     return out
 
 
-def config_of(wl: I.Workload, world: int) -> dict:
+def config_of(wl: I.Workload, world: int, opts=None) -> dict:
     """The `config` object, identical in both arms."""
+    o = opts or NO_OPTIONS
     return {"workload": wl.name, "B": wl.B, "M": wl.M, "d": wl.d, "V": wl.V, "mode": "judge_or_standard",
+            "rule": o["rule"] if o["rule"] == "sampling" else "top-%d" % o["top_k"],
+            "norm": "rms" if o["rms_eps"] else "none",
             "l2": "not flushed between calls: inputs larger than L2 (W is %.2f GB, L2 126 MB)" %
                   (wl.V * wl.d * (1 if wl.dtype == "fp8" else 2) / 1e9),
             "parallelism": "replicas only" if world > 1 else "single GPU"}
 
 
-def run_reference(args, wl) -> None:
+def run_reference(args, wl, opts) -> None:
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -314,15 +317,15 @@ def run_reference(args, wl) -> None:
     # the workload; only when K steps of even one sequence would run for more than ~5 minutes are
     # they cut down, and the line says so
     t0 = time.perf_counter()
-    oracle_step(inp, 0, [0])
+    oracle_step(inp, 0, [0], opts)
     one = time.perf_counter() - t0
     steps = int(max(1, min(args.steps, 300.0 / max(one, 1e-3))))
     warmup = int(max(2, min(args.warmup, 30.0 / max(one, 1e-3))))   # the call above + time_oracle's sizing call + ...
-    r = time_oracle(inp, steps, budget_s=max(60.0, one * steps), extra_warmup=warmup - 2)
+    r = time_oracle(inp, steps, budget_s=max(60.0, one * steps), extra_warmup=warmup - 2, opts=opts)
     line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": r["seconds"] / steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": config_of(wl, 1),
+            "data": "synthetic", "config": config_of(wl, 1, opts),
             "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
             "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -475,8 +478,8 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=3, help="workload id of the headline line (1..4); default: the "
-                    "405B-shaped head, the largest single-GPU configuration")
+    ap.add_argument("--config", default="3", help="workload of the headline line: an id 1..4, optionally followed by "
+                    "the option letters of --others; default: the 405B-shaped head, the largest single-GPU configuration")
     ap.add_argument("--others", default="2,1,4,3f,4f", help="comma list of further workloads summarised in the same "
                     "line: an id, then f = FP8 E4M3 head, g / k = greedy / top-5 rule, n = RMSNorm ahead of the head")
     ap.add_argument("--record-traffic", nargs="+", metavar="WORKLOAD=CSV[,CSV]", help="rewrite profiles/ncu_traffic.json "
@@ -490,12 +493,15 @@ def main() -> None:
         record_traffic(args.record_traffic)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    wl = I.CONFIGS[args.config]
-    if args.fp8:
-        wl = wl.scaled(wl.name + "-fp8", dtype="fp8")
+    tok = args.config.strip()
+    if args.fp8 and "f" not in tok:
+        tok = re.sub(r"^(\d+)", r"\1f", tok)
+    wl, opts = parse_workload_token(tok)
+    if wl is None:
+        ap.error("--config %s: not a workload" % args.config)
 
     if args.impl == "reference":
-        run_reference(args, wl)
+        run_reference(args, wl, opts)
         return
 
     import torch
@@ -512,7 +518,7 @@ def main() -> None:
         torch.distributed.init_process_group("nccl", device_id=device)
 
     peaks, which = load_peaks()
-    res = measure_workload(wl, args, torch, jd, device, data_seed=rank, sample_clocks=True)
+    res = measure_workload(wl, args, torch, jd, device, data_seed=rank, sample_clocks=True, opts=opts)
 
     # max over ranks of the timed region, sum of the units
     total_ms, e2e_s = max_over_ranks([res["total_ms"], res["e2e_s"]], device, args.dist)
@@ -558,14 +564,14 @@ def main() -> None:
         cpu, parity = None, None
         log("workloads done; CPU baseline")
         if not args.no_cpu_baseline:
-            c = time_oracle(res["inp"], 1)
+            c = time_oracle(res["inp"], 1, opts=opts)
             cpu = {k: c[k] for k in ("value", "unit", "cores", "kind", "sample")}
-            parity = parity_of(wl, res["out0"], c["first"])
+            parity = parity_of(wl, res["out0"], c["first"], rule=opts["rule"])
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "fp8" if wl.dtype == "fp8" else "bf16", "data": "synthetic",
-            "config": config_of(wl, world),
+            "config": config_of(wl, world, opts),
             "variant": VARIANT_NAMES.get(res["variant"], "?"), "mean_accept_len": res["mean_accept"],
             "calls_per_s": world * K / (total_ms * 1e-3),
             "median_ms_per_step": res["median_ms"],

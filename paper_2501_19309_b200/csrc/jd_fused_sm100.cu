@@ -484,96 +484,8 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       if (tid == 0) mbar_arrive(smem_u32(&ms.drained));
     }
 
-    // (b) while W streams: draft-row statistics over this CTA's vocabulary slice, judge dots
-    if (fp.dl_flag != nullptr) {   // draft logits still in flight: wait for the copy stream's signal
-      if (tid == 0) {
-        bool arrived = false;
-        for (unsigned it = 0; it < kSpinLimit / 4 && !arrived; ++it) {
-          unsigned v;
-          asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(fp.dl_flag) : "memory");
-          arrived = (v == fp.dl_epoch);
-          if (!arrived) {
-            if (*abort_flag) break;
-            __nanosleep(100);
-          }
-        }
-        if (!arrived) {
-          *abort_flag = 1;
-          report(JD_ERR_TIMEOUT);
-        }
-      }
-      epi_sync();
-    }
-    const int v_lo = t0 * kVocabTile, v_hi = min(V, (t0 + T) * kVocabTile);
-    const bool vec4 = cp.dl_vec4 != 0;   // rows start on 16-byte boundaries only then
-    for (int bm = warp; bm < (kSampleOnly ? 0 : BM); bm += 4) {
-      const float* row = cp.draft_logits + (size_t)bm * V;
-      float m = -INFINITY, s = 0.f;
-      if (vec4) {
-        // eight 128-entry tiles per pass: all loads of the pass are issued before any arithmetic
-        for (int i0 = 0; i0 < T; i0 += 8) {
-          float4 x[8];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int v = v_lo + (i0 + u) * kVocabTile + lane * 4;
-            x[u] = (i0 + u < T && v < V) ? __ldcg(reinterpret_cast<const float4*>(row + v))
-                                         : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-          }
-          float mm = -INFINITY;
-#pragma unroll
-          for (int u = 0; u < 8; ++u) mm = fmaxf(mm, fmaxf(fmaxf(x[u].x, x[u].y), fmaxf(x[u].z, x[u].w)));
-          const float mn = fmaxf(m, mm);
-          if (mn == -INFINITY) continue;
-          float acc = 0.f;
-          const float off = mn * kLog2e;
-#pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            acc += exp2f(fmaf(x[u].x, kLog2e, -off)) + exp2f(fmaf(x[u].y, kLog2e, -off));
-            acc += exp2f(fmaf(x[u].z, kLog2e, -off)) + exp2f(fmaf(x[u].w, kLog2e, -off));
-          }
-          s = s * __expf(m - mn) + acc;
-          m = mn;
-        }
-      } else {
-        for (int v = v_lo + lane; v < v_hi; v += 32) {
-          const float xv = __ldcg(row + v);
-          if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
-          else if (xv != -INFINITY) s += __expf(xv - m);
-        }
-      }
-      ms_warp_reduce(m, s);
-      if (lane == 0) {
-        ws.qpart_max[(size_t)bm * G + cta] = m;
-        ws.qpart_sum[(size_t)bm * G + cta] = s;
-        const int b = bm / M, j = bm % M;
-        const int x = ms.x_row[b * (M + 1) + j];
-        if (x >= v_lo && x < v_hi) ws.qgath[bm] = __ldcg(row + x);
-      }
-    }
-    for (int bm = cta * 4 + warp; bm < (kSampleOnly ? 0 : BM); bm += G * 4) {
-      const int b = bm / M, j = bm % M;
-      const uint4* h4 = reinterpret_cast<const uint4*>(H + ((size_t)b * (M + 1) + j + 1) * cp.d);
-      const uint4* w4 = reinterpret_cast<const uint4*>(wj);
-      float acc = 0.f;
-      for (int k = lane; k < cp.d / 8; k += 32) {
-        const uint4 hv = __ldg(h4 + k), wv = __ldg(w4 + k);
-        const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
-        const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float2 a = __bfloat1622float2(hp[e]), c = __bfloat1622float2(wp[e]);
-          acc = fmaf(a.x, c.x, acc);
-          acc = fmaf(a.y, c.y, acc);
-        }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (lane == 0) ws.judge_logit[bm] = acc;
-    }
-
-    JD_STAMP(1);
-    // (c)-(e) row statistics, in one or two phases. Phase 1 covers the tiles of the last sweep and
-    // starts when the whole accumulation is complete. A CTA that ran an early sweep (T_early > 0)
+    // (b)-(e) draft statistics and judge dots, then the row statistics in one or two phases. Phase 1
+    // covers the tiles of the last sweep and starts when the whole accumulation is complete. A CTA that ran an early sweep (T_early > 0)
     // first takes, in phase 0, the statistics of the early tiles while the last sweep still streams,
     // and merges the two (max, sum exp) pairs per row at the end.
     if constexpr (kSampleOnly) {
@@ -587,7 +499,104 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
       }
       epi_sync();
     }
-    for (int ph = (T_early > 0 ? 0 : 1); ph < 2; ++ph) {
+    // Order of the steps: (b), then phase 0 (if there is an early sweep), then phase 1. A call whose draft
+    // logits are still on their way from the host runs phase 0 first, so that the copy has the early
+    // sweep's time to land before anything waits for it.
+    const bool defer_b = fp.dl_flag != nullptr && T_early > 0;
+    for (int step = 0; step < 3; ++step) {
+      const int ph = defer_b ? (step == 0 ? 0 : (step == 1 ? -1 : 1)) : step - 1;
+      if (ph < 0) {
+      // (b) while W streams: draft-row statistics over this CTA's vocabulary slice, judge dots
+      if (fp.dl_flag != nullptr) {   // draft logits still in flight: wait for the copy stream's signal
+        if (tid == 0) {
+          bool arrived = false;
+          for (unsigned it = 0; it < kSpinLimit / 4 && !arrived; ++it) {
+            unsigned v;
+            asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(fp.dl_flag) : "memory");
+            arrived = (v == fp.dl_epoch);
+            if (!arrived) {
+              if (*abort_flag) break;
+              __nanosleep(100);
+            }
+          }
+          if (!arrived) {
+            *abort_flag = 1;
+            report(JD_ERR_TIMEOUT);
+          }
+        }
+        epi_sync();
+      }
+      const int v_lo = t0 * kVocabTile, v_hi = min(V, (t0 + T) * kVocabTile);
+      const bool vec4 = cp.dl_vec4 != 0;   // rows start on 16-byte boundaries only then
+      for (int bm = warp; bm < (kSampleOnly ? 0 : BM); bm += 4) {
+        const float* row = cp.draft_logits + (size_t)bm * V;
+        float m = -INFINITY, s = 0.f;
+        if (vec4) {
+          // eight 128-entry tiles per pass: all loads of the pass are issued before any arithmetic
+          for (int i0 = 0; i0 < T; i0 += 8) {
+            float4 x[8];
+  #pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int v = v_lo + (i0 + u) * kVocabTile + lane * 4;
+              x[u] = (i0 + u < T && v < V) ? __ldcg(reinterpret_cast<const float4*>(row + v))
+                                           : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            }
+            float mm = -INFINITY;
+  #pragma unroll
+            for (int u = 0; u < 8; ++u) mm = fmaxf(mm, fmaxf(fmaxf(x[u].x, x[u].y), fmaxf(x[u].z, x[u].w)));
+            const float mn = fmaxf(m, mm);
+            if (mn == -INFINITY) continue;
+            float acc = 0.f;
+            const float off = mn * kLog2e;
+  #pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              acc += exp2f(fmaf(x[u].x, kLog2e, -off)) + exp2f(fmaf(x[u].y, kLog2e, -off));
+              acc += exp2f(fmaf(x[u].z, kLog2e, -off)) + exp2f(fmaf(x[u].w, kLog2e, -off));
+            }
+            s = s * __expf(m - mn) + acc;
+            m = mn;
+          }
+        } else {
+          for (int v = v_lo + lane; v < v_hi; v += 32) {
+            const float xv = __ldcg(row + v);
+            if (xv > m) { s = s * __expf(m - xv) + 1.f; m = xv; }
+            else if (xv != -INFINITY) s += __expf(xv - m);
+          }
+        }
+        ms_warp_reduce(m, s);
+        if (lane == 0) {
+          ws.qpart_max[(size_t)bm * G + cta] = m;
+          ws.qpart_sum[(size_t)bm * G + cta] = s;
+          const int b = bm / M, j = bm % M;
+          const int x = ms.x_row[b * (M + 1) + j];
+          if (x >= v_lo && x < v_hi) ws.qgath[bm] = __ldcg(row + x);
+        }
+      }
+      for (int bm = cta * 4 + warp; bm < (kSampleOnly ? 0 : BM); bm += G * 4) {
+        const int b = bm / M, j = bm % M;
+        const uint4* h4 = reinterpret_cast<const uint4*>(H + ((size_t)b * (M + 1) + j + 1) * cp.d);
+        const uint4* w4 = reinterpret_cast<const uint4*>(wj);
+        float acc = 0.f;
+        for (int k = lane; k < cp.d / 8; k += 32) {
+          const uint4 hv = __ldg(h4 + k), wv = __ldg(w4 + k);
+          const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+          const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+  #pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 a = __bfloat1622float2(hp[e]), c = __bfloat1622float2(wp[e]);
+            acc = fmaf(a.x, c.x, acc);
+            acc = fmaf(a.y, c.y, acc);
+          }
+        }
+  #pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) ws.judge_logit[bm] = acc;
+      }
+
+        JD_STAMP(1);
+        continue;
+      }
+      if (ph == 0 && T_early == 0) continue;
       if (tid == 0 && ok && (ph == 0 || T > n_ovf)) mbar_wait(smem_u32(&ms.acc_full[ph]), 0u, abort_flag);
       epi_sync();
       tc_fence_after();

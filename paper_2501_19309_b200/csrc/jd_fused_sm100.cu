@@ -667,6 +667,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             }
           }
         }
+        if (ph == 0) JD_STAMP(14);
         continue;
       }
 
@@ -758,6 +759,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         }
       }
       epi_sync();
+      if (ph == 0) JD_STAMP(14);
     }
     JD_STAMP(3);
     if constexpr (!kSampleOnly) {
@@ -1009,6 +1011,12 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     // slice contains T = u * total (same arithmetic in every CTA, so every CTA agrees) ...
     if (ok && draw) {
       const int per = (G + 31) / 32;   // lane l owns CTAs [l*per, (l+1)*per), per <= 8
+      double nx[8];                    // the next sequence's masses, fetched while this one is searched
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int c = lane * per + u;
+        nx[u] = (warp < cp.B && u < per && c < G) ? __ldcg(ws.mass_r + (size_t)warp * G + c) : 0.0;
+      }
       for (int b = warp; b < cp.B; b += 4) {
         const double* mass = ws.mass_r + (size_t)b * G;
         double mc[8];
@@ -1016,8 +1024,9 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           const int c = lane * per + u;
-          mc[u] = (u < per && c < G) ? __ldcg(mass + c) : 0.0;
+          mc[u] = nx[u];
           chunk += mc[u];
+          if (b + 4 < cp.B) nx[u] = (u < per && c < G) ? __ldcg(mass + (size_t)4 * G + c) : 0.0;
         }
         double total = warp_sum_double(chunk);
         int use_p = 0;

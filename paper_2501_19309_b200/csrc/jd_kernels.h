@@ -43,7 +43,8 @@ bool batched_configure();
 // kMaxCtas x kPhaseStampSlots global-timer values in ns, slot = 0 start of the epilogue, 1 draft statistics and
 // judge dots done, 12 early sweep complete, 2 stream complete, 3 row statistics done, 4 barrier 1 passed,
 // 5 fold done, 6 barrier 2 passed, 7 decisions done, 8 sampling masses done, 9 barrier 3 passed, 10 owner
-// found, 11 end of the epilogue, 13 the previous launch's slot 11.
+// found, 11 end of the epilogue, 13 the previous launch's slot 11, 14 statistics (sample-only mode: masses) of the
+// early tiles done.
 constexpr int kPhaseStampSlots = 16;
 bool read_phase_stamps(unsigned long long* host_out);
 void launch_timeout_probe(const Workspace& ws, unsigned limit, cudaStream_t st);

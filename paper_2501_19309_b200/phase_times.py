@@ -6,7 +6,7 @@ thread 0 of every CTA records the GPU's global timer at the phase boundaries of 
 Usage: ``python -m paper_2501_19309_b200.phase_times [workloads, default 1,2,3; a trailing f = FP8 head]``
 
 For every workload (the synthetic shapes of ``inputs.CONFIGS``) it runs batches of back-to-back calls,
-reads the stamps of the last call of each batch and prints, per phase, the minimum / median / maximum over
+reads the stamps of the last call of each batch (of a batched-variant call: those of its second pass) and prints, per phase, the minimum / median / maximum over
 the CTAs of the median over batches, in microseconds from the first CTA's start, then the distance between
 one call's last stamp and the next call's first, and the time per call of a longer back-to-back loop.
 """
@@ -26,7 +26,7 @@ from . import jd  # noqa: E402
 
 CTAS, SLOTS = 256, 16
 PHASES = [(0, "start of the epilogue"), (1, "draft statistics + judge dots done"), (12, "early sweep complete"),
-          (2, "W stream complete"), (3, "row statistics done"), (4, "barrier 1 passed"), (5, "fold done"),
+          (14, "early tiles' statistics done"), (2, "W stream complete"), (3, "row statistics done"), (4, "barrier 1 passed"), (5, "fold done"),
           (6, "barrier 2 passed"), (7, "decisions done"), (8, "sampling masses done"), (9, "barrier 3 passed"),
           (10, "owner found"), (11, "end of the epilogue")]
 
@@ -58,7 +58,9 @@ def main() -> None:
         ver = jd.Verifier(wl.B, wl.M, wl.d, wl.V, "fp8" if fp8 else "bf16", 0)
         ver.set_head(W, w, inp.b_judge, w_scale=ws)
         out = ver.alloc_outputs(wl.B, wl.M)
-        args = [ver.make_args(H, x, dl, inp.tau, s, "judge_or_standard", out=out, variant="fused")[0] for s in range(8)]
+        # more than 96 rows: the batched variant, whose second pass is the fused kernel in its sample-only mode
+        variant = "fused" if wl.B * (wl.M + 1) <= 96 else "auto"
+        args = [ver.make_args(H, x, dl, inp.tau, s, "judge_or_standard", out=out, variant=variant)[0] for s in range(8)]
         stream = torch.cuda.current_stream(dev)
 
         def run(n):
@@ -82,7 +84,7 @@ def main() -> None:
         print("== %s: us from the first CTA's start (min / median / max over %d CTAs)" % (wl.name, n_ctas))
         for k, name in PHASES:
             col = r[:, k]
-            if k == 12 and (col <= 0).all():
+            if (col <= 0).all():      # a phase this call does not have (its slot still holds an older or no stamp)
                 continue
             print("  %-38s %8.1f %8.1f %8.1f" % (name, col.min(), np.median(col), col.max()))
         print("  %-38s %8.1f" % ("next call's first stamp after the last", float(np.median(gaps))))

@@ -164,6 +164,8 @@ size_t carve(const jd_config_t& c, char* base, Workspace* ws, size_t* guard_off 
   w.argidx = (int*)take(maxR * 4);
   w.part_idx = (int*)take(maxR * np * 4);
   w.cand_ref = (float*)take(maxR * 4);
+  w.own_i = (int*)take(maxB * 2 * 4);
+  w.own_d = (double*)take(maxB * 2 * 8);
   w.status = (unsigned*)take(512);   // status word and, 256 bytes on, the barrier counters: one memset per call
   w.barrier = w.status ? w.status + 64 : nullptr;
   char* flag = take(256);   // word 0: arrival flag of a host-buffer call's draft logits; outside the per-call memset

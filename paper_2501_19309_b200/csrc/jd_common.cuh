@@ -47,6 +47,9 @@ struct Workspace {
   int* part_idx;       // [maxR][np] top-K rule: per-CTA argmax candidates (fused variant); lowest token id
                        //            that attains the tile's maximum, per vocabulary tile (batched variant)
   float* cand_ref;     // [maxR] top-K rule, batched variant: L[row, x_j] computed ahead of the GEMM pass
+  int* own_i;          // [maxB][2] second pass of the batched variant: CTA that owns each sequence's draw, and whether
+                       //           the draw falls back to p (identically zero residual)
+  double* own_d;       // [maxB][2] same: mass in front of the owning CTA's slice (< 0: beyond the total), and T
   __nv_bfloat16* h_sel;  // [maxB][d] selected rows of H gathered for the batched variant's second pass
   unsigned* status;    // [1] device status word: jd_status_t of the first device-side problem in bits 0-7; bits 8-31 a
                        //     call tag when the fused kernel wrote it (see kCallCounter), 0 when another kernel did

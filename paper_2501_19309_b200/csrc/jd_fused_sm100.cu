@@ -31,6 +31,8 @@
 //   every CTA runs the tests and the prefix rule (identical results), then computes its slice
 //   of the sampling mass of each sequence's selected row                        -> barrier 3
 //   the CTA whose slice contains T = u * total mass locates the token.
+// (Sample-only mode skips the first two meetings and uses the first counter once more after the third: the
+// searches for the owning CTAs of its up to 96 sequences are dealt out over the grid and exchanged there.)
 // The barriers are counters in global memory, legal because the launch is cooperative (all
 // CTAs co-resident); every wait in the kernel is bounded and reports JD_ERR_TIMEOUT.
 #include <cooperative_groups.h>
@@ -1011,13 +1013,18 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     // slice contains T = u * total (same arithmetic in every CTA, so every CTA agrees) ...
     if (ok && draw) {
       const int per = (G + 31) / 32;   // lane l owns CTAs [l*per, (l+1)*per), per <= 8
+      // Sample-only mode (up to 96 sequences): the searches are dealt out over the grid, one per warp, and
+      // their results exchanged through global memory behind one more grid barrier; otherwise every CTA
+      // searches for every sequence itself.
+      const int b_first = kSampleOnly ? cta + G * warp : warp;
+      const int b_step = kSampleOnly ? 4 * G : 4;
       double nx[8];                    // the next sequence's masses, fetched while this one is searched
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int c = lane * per + u;
-        nx[u] = (warp < cp.B && u < per && c < G) ? __ldcg(ws.mass_r + (size_t)warp * G + c) : 0.0;
+        nx[u] = (b_first < cp.B && u < per && c < G) ? __ldcg(ws.mass_r + (size_t)b_first * G + c) : 0.0;
       }
-      for (int b = warp; b < cp.B; b += 4) {
+      for (int b = b_first; b < cp.B; b += b_step) {
         const double* mass = ws.mass_r + (size_t)b * G;
         double mc[8];
         double chunk = 0.0;
@@ -1026,7 +1033,7 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           const int c = lane * per + u;
           mc[u] = nx[u];
           chunk += mc[u];
-          if (b + 4 < cp.B) nx[u] = (u < per && c < G) ? __ldcg(mass + (size_t)4 * G + c) : 0.0;
+          if (b + b_step < cp.B) nx[u] = (u < per && c < G) ? __ldcg(mass + (size_t)b_step * G + c) : 0.0;
         }
         double total = warp_sum_double(chunk);
         int use_p = 0;
@@ -1078,10 +1085,38 @@ fused_verify_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
           owner_prefix = -1.0;
         }
         if (lane == 0) {
-          ms.own_cta[b] = owner;
-          ms.own_prefix[b] = owner_prefix;
-          ms.own_T[b] = Tt;
-          ms.own_usep[b] = use_p;
+          if constexpr (kSampleOnly) {
+            ws.own_i[2 * b] = owner;
+            ws.own_i[2 * b + 1] = use_p;
+            ws.own_d[2 * b] = owner_prefix;
+            ws.own_d[2 * b + 1] = Tt;
+          } else {
+            ms.own_cta[b] = owner;
+            ms.own_prefix[b] = owner_prefix;
+            ms.own_T[b] = Tt;
+            ms.own_usep[b] = use_p;
+          }
+        }
+      }
+    }
+    if constexpr (kSampleOnly) {
+      // exchange of the search results: the counter of barrier 1, which this mode does not use otherwise
+      __threadfence();
+      epi_sync();
+      if (tid == 0) {
+        if (!ok || !grid_arrive_and_wait(bar + 0, (unsigned)G, abort_flag)) {
+          *abort_flag = 1;
+          report(JD_ERR_TIMEOUT);
+        }
+      }
+      epi_sync();
+      ok = (*abort_flag == 0);
+      if (ok) {
+        for (int b = tid; b < cp.B; b += 128) {
+          ms.own_cta[b] = __ldcg(ws.own_i + 2 * b);
+          ms.own_usep[b] = __ldcg(ws.own_i + 2 * b + 1);
+          ms.own_prefix[b] = __ldcg(ws.own_d + 2 * b);
+          ms.own_T[b] = __ldcg(ws.own_d + 2 * b + 1);
         }
       }
     }
@@ -1328,6 +1363,9 @@ int run_fused(const CallParams& cp, const Workspace& ws, const CUtensorMap& tmW,
   // before at 80 (cfg2) and is even with a single sweep at 32 rows and d = 16384 (cfg3): on wherever the sweep
   // over d is long enough to hide something (32 k-steps) or the statistics passes are long (48 padded rows).
   fp.late_tiles = (sample_only || plan.n_pad >= 48 || fp.num_kb >= 32) ? 1 : 0;
+  // Sample-only mode with an FP8 head and many sequences: one tile of codes streams in half the time the
+  // masses of the early tiles take, so two tiles are left for the late sweep.
+  if (sample_only && w_scale_fp8 != nullptr && plan.n_pad >= 48) fp.late_tiles = 2;
   fp.off_h = kMiscBytes;
   fp.off_ovf = fp.off_h + plan.h_stages * plan.n_pad * 128;
   const int n_ovf = plan.max_tiles - plan.tmem_tiles;

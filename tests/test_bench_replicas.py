@@ -58,3 +58,21 @@ def test_roofline_bound_selection():
     assert r4["bound"] == "tensor" and abs(r4["achieved"] - 2 * 1088 * 128256 * 8192 / 2e-3 / 1e12) < 1e-6
     line = json.dumps(r4)
     assert "traffic" in line
+
+
+def test_workload_tokens_of_the_bench():
+    """An id, then f = FP8 head, g / k = greedy / top-5 rule, n = RMSNorm; anything else is no workload."""
+    sys.path.insert(0, ROOT)
+    import bench
+    wl, o = bench.parse_workload_token("3")
+    assert wl.name == "cfg3-405B-head" and wl.dtype == "bf16" and o == bench.NO_OPTIONS
+    wl, o = bench.parse_workload_token("4f")
+    assert wl.name == "cfg4-batched-fp8" and wl.dtype == "fp8" and o["rule"] == "sampling" and o["rms_eps"] is None
+    wl, o = bench.parse_workload_token("2gn")
+    assert wl.name == "cfg2-70B-head-greedy-rmsnorm" and (o["rule"], o["top_k"]) == ("topk", 1) and o["rms_eps"] > 0
+    wl, o = bench.parse_workload_token("1fk")
+    assert wl.dtype == "fp8" and (o["rule"], o["top_k"]) == ("topk", 5) and (wl.B, wl.M, wl.d) == (1, 8, 4096)
+    for bad in ("", "9", "3x", "g3", "3gk", "3nf"):
+        assert bench.parse_workload_token(bad) == (None, None)
+    cfg = bench.config_of(*bench.parse_workload_token("4g")[:1], 1, bench.parse_workload_token("4g")[1])
+    assert cfg["rule"] == "top-1" and cfg["norm"] == "none" and cfg["workload"] == "cfg4-batched-greedy"

@@ -320,7 +320,7 @@ def run_reference(args, wl, opts) -> None:
     oracle_step(inp, 0, [0], opts)
     one = time.perf_counter() - t0
     steps = int(max(1, min(args.steps, 300.0 / max(one, 1e-3))))
-    warmup = int(max(2, min(args.warmup, 30.0 / max(one, 1e-3))))   # the call above + time_oracle's sizing call + ...
+    warmup = int(max(2, min(args.warmup, 60.0 / max(one, 1e-3))))   # the call above + time_oracle's sizing call + ...
     r = time_oracle(inp, steps, budget_s=max(60.0, one * steps), extra_warmup=warmup - 2, opts=opts)
     line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": r["seconds"] / steps * 1e3,
